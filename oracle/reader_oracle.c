@@ -1,0 +1,344 @@
+/*
+ * reader_oracle.c -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, fp64 CPU statement of what one batched tree-verification
+ * step of READER-style lossless speculative decoding computes.  It exists so
+ * that the CUDA library can be checked against something that can be read
+ * side by side with the paper.  Nothing in the product path may call it, and
+ * it shares no code, header, table or helper with the CUDA sources.
+ *
+ * What each function follows:
+ *   oracle_ancestor_matrix  Sec. 3.2 ("Tree Decoding"): the decoding mask M
+ *                           with M_ij = 1 iff node i is an ancestor of node j.
+ *   oracle_verify_attn      Sec. 3.2: scaled dot-product attention of the
+ *                           gamma tree queries against the s cached keys plus
+ *                           the gamma tree keys under that mask.
+ *   oracle_argmax /         Algorithm 5 (Verify) step 2 and Appendix C,
+ *   oracle_accept           invariants 1-3 and the deterministic theorem:
+ *                           compare the base model's greedy choice with the
+ *                           drafted tokens, keep the longest consistent prefix.
+ *   oracle_kv_commit        Sec. 4.3 and Algorithm 4 (KVCacheRearrange): the
+ *                           accepted entries are concatenated tightly behind
+ *                           the committed cache, per sample.
+ *
+ * Readings taken where the paper is silent (each is listed in the design
+ * document as well):
+ *   - a node always sees itself (the mask is made reflexive);
+ *   - node 0 is the root, parent[0] = -1 and 0 <= parent[j] < j;
+ *   - the root is the last committed token: it is always accepted, so the
+ *     accepted length counts it and is >= 1;
+ *   - argmax ties go to the lowest token id; a NaN never wins a comparison
+ *     and a NaN in slot 0 counts as -infinity;
+ *   - when several consistent paths have the same length the one ending at
+ *     the lowest node index is returned; equal sibling tokens are all
+ *     explored;
+ *   - nodes deeper than max_path are not candidates (their ancestor at that
+ *     depth still is).
+ *
+ * Pins (tests/test_oracle_*.py, run without a GPU): chain tree == causal
+ * attention and single node == decode attention against torch's CPU
+ * scaled_dot_product_attention; closed forms (uniform keys -> mean of V, one
+ * dominant key -> that V); probabilities sum to one; split-and-merge algebra;
+ * sibling-order and page-permutation invariance; exhaustive acceptance on
+ * all trees with <= 6 nodes against an independently written accepted-set
+ * propagation; Eq. 1 statistics; the deterministic-losslessness loop.
+ * Absolute attention values on random inputs beyond those pins: parity
+ * unpinned (the paper prints no worked numeric example).
+ *
+ * Layouts (row-major, last index fastest):
+ *   q, out        [B][T][Hq][D]        k_tree, v_tree  [B][T][Hkv][D]
+ *   k_pool,v_pool [num_pages][Hkv][P][D]
+ *   page_table    [B][max_pages]       seq_lens [B]    parent [B][T]
+ * bf16 values travel as uint16_t bit patterns; widening to double is exact.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum {
+    ORACLE_OK = 0,
+    ORACLE_BAD_TREE = 2,
+    ORACLE_CAPACITY = 3,
+    ORACLE_BAD_PAGE = 8
+};
+
+static double bf16_bits_to_double(uint16_t bits)
+{
+    uint32_t u = (uint32_t)bits << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* Node numbering rule: one root at index 0, every other parent precedes its child. */
+int oracle_tree_is_valid(const int32_t *parent, int n_nodes)
+{
+    if (n_nodes < 1 || parent[0] != -1) return 0;
+    for (int j = 1; j < n_nodes; ++j)
+        if (parent[j] < 0 || parent[j] >= j) return 0;
+    return 1;
+}
+
+/* Sec. 3.2: M[i][j] = 1 iff node i is an ancestor of node j (here: or i == j).
+ * Found by walking from j towards the root.  M is [T][T], row i, column j. */
+void oracle_ancestor_matrix(const int32_t *parent, int n_nodes, uint8_t *M)
+{
+    memset(M, 0, (size_t)n_nodes * n_nodes);
+    for (int j = 0; j < n_nodes; ++j)
+        for (int i = j; i >= 0; i = parent[i])
+            M[(size_t)i * n_nodes + j] = 1;
+}
+
+/* Number of nodes on the path root..j (root has level 1). */
+void oracle_levels(const int32_t *parent, int n_nodes, int32_t *level)
+{
+    for (int j = 0; j < n_nodes; ++j) {
+        int c = 0;
+        for (int i = j; i >= 0; i = parent[i]) ++c;
+        level[j] = c;
+    }
+}
+
+/*
+ * Sec. 3.2 attention.  For sequence b, node j, query head h (KV head h / G):
+ * the visible keys are the committed positions 0..L_b-1, reached through the
+ * page table, and the tree nodes on the path root..j.  Scores, softmax and
+ * the weighted sum of values are all fp64.
+ *
+ * probs (nullable) receives the softmax weights, [B][T][Hq][probs_stride]:
+ * committed position p at column p, tree node i at column L_b + i, zero for
+ * keys that are not visible.  lse (nullable) receives log(sum(exp(score))).
+ * status[b] != 0 leaves that sequence's outputs at zero.
+ */
+void oracle_verify_attn(const uint16_t *q, const uint16_t *k_tree, const uint16_t *v_tree,
+                        const uint16_t *k_pool, const uint16_t *v_pool,
+                        int num_pages, int page_size, int n_kv_heads, int head_dim,
+                        const int32_t *page_table, int max_pages, const int32_t *seq_lens,
+                        const int32_t *parent, int batch, int n_nodes, int n_q_heads,
+                        double scale, double *out, double *lse, double *probs,
+                        int64_t probs_stride, int32_t *status)
+{
+    const int G = n_q_heads / n_kv_heads;
+    const int D = head_dim;
+
+    for (int b = 0; b < batch; ++b) {
+        int st = ORACLE_OK;
+        const int L = seq_lens[b];
+        if (!oracle_tree_is_valid(parent + (size_t)b * n_nodes, n_nodes)) st = ORACLE_BAD_TREE;
+        else if (L < 0 || (int64_t)L > (int64_t)max_pages * page_size) st = ORACLE_CAPACITY;
+        else
+            for (int p = 0; p * page_size < L; ++p) {
+                int32_t pg = page_table[(size_t)b * max_pages + p];
+                if (pg < 0 || pg >= num_pages) st = ORACLE_BAD_PAGE;
+            }
+        status[b] = st;
+    }
+
+    memset(out, 0, sizeof(double) * (size_t)batch * n_nodes * n_q_heads * D);
+    if (lse) memset(lse, 0, sizeof(double) * (size_t)batch * n_nodes * n_q_heads);
+    if (probs) memset(probs, 0, sizeof(double) * (size_t)batch * n_nodes * n_q_heads * probs_stride);
+
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < batch; ++b) {
+        for (int h = 0; h < n_q_heads; ++h) {
+            if (status[b] != ORACLE_OK) continue;
+            const int L = seq_lens[b];
+            const int hk = h / G;
+            const int32_t *par = parent + (size_t)b * n_nodes;
+            double *score = (double *)malloc(sizeof(double) * (size_t)(L + n_nodes));
+            const uint16_t **kptr = (const uint16_t **)malloc(sizeof(void *) * (size_t)(L + n_nodes));
+            const uint16_t **vptr = (const uint16_t **)malloc(sizeof(void *) * (size_t)(L + n_nodes));
+            int64_t *col = (int64_t *)malloc(sizeof(int64_t) * (size_t)(L + n_nodes));
+
+            for (int j = 0; j < n_nodes; ++j) {
+                const size_t row = ((size_t)b * n_nodes + j) * n_q_heads + h;
+                const uint16_t *qrow = q + row * D;
+
+                /* gather the visible keys */
+                int n = 0;
+                for (int pos = 0; pos < L; ++pos) {
+                    const int32_t pg = page_table[(size_t)b * max_pages + pos / page_size];
+                    const size_t at = (((size_t)pg * n_kv_heads + hk) * page_size + pos % page_size) * D;
+                    kptr[n] = k_pool + at;
+                    vptr[n] = v_pool + at;
+                    col[n] = pos;
+                    ++n;
+                }
+                for (int i = j; i >= 0; i = par[i]) {
+                    const size_t at = (((size_t)b * n_nodes + i) * n_kv_heads + hk) * D;
+                    kptr[n] = k_tree + at;
+                    vptr[n] = v_tree + at;
+                    col[n] = (int64_t)L + i;
+                    ++n;
+                }
+
+                /* scores */
+                double smax = -INFINITY;
+                for (int t = 0; t < n; ++t) {
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d)
+                        dot += bf16_bits_to_double(qrow[d]) * bf16_bits_to_double(kptr[t][d]);
+                    score[t] = scale * dot;
+                    if (score[t] > smax) smax = score[t];
+                }
+                /* softmax */
+                double denom = 0.0;
+                for (int t = 0; t < n; ++t) {
+                    score[t] = exp(score[t] - smax);
+                    denom += score[t];
+                }
+                /* weighted values */
+                double *orow = out + row * D;
+                for (int t = 0; t < n; ++t) {
+                    const double p = score[t] / denom;
+                    if (probs) probs[row * probs_stride + col[t]] = p;
+                    for (int d = 0; d < D; ++d)
+                        orow[d] += p * bf16_bits_to_double(vptr[t][d]);
+                }
+                if (lse) lse[row] = smax + log(denom);
+            }
+            free(score);
+            free((void *)kptr);
+            free((void *)vptr);
+            free(col);
+        }
+    }
+}
+
+/* Greedy policy of Appendix C with a fixed tie-break: first index of the maximum. */
+int32_t oracle_argmax_row(const float *row, int64_t vocab)
+{
+    float best = row[0];
+    int64_t at = 0;
+    if (isnan(best)) best = -INFINITY;
+    for (int64_t v = 1; v < vocab; ++v)
+        if (row[v] > best) {
+            best = row[v];
+            at = v;
+        }
+    return (int32_t)at;
+}
+
+void oracle_argmax(const float *logits, int64_t rows, int64_t vocab, int32_t *target)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        target[r] = oracle_argmax_row(logits + r * vocab, vocab);
+}
+
+/*
+ * Algorithm 5 step 2 / Appendix C invariant 2, by brute force: every node e
+ * is tried as the end of a root-to-e path; the path is consistent when every
+ * non-root node u on it carries the token the base model picks after its
+ * parent, tok[u] == target[parent[u]].  The longest consistent path wins,
+ * lowest e among equals.  bonus = target[e] is the token invariant 3 commits
+ * after the last accepted one.  path is padded with -1.
+ */
+void oracle_accept(const int32_t *parent, const int32_t *tok, const int32_t *target,
+                   int batch, int n_nodes, int max_path,
+                   int32_t *path, int32_t *n_acc, int32_t *bonus, int32_t *status)
+{
+    for (int b = 0; b < batch; ++b) {
+        const int32_t *par = parent + (size_t)b * n_nodes;
+        const int32_t *tk = tok + (size_t)b * n_nodes;
+        const int32_t *tg = target + (size_t)b * n_nodes;
+        int32_t *pth = path + (size_t)b * max_path;
+        for (int k = 0; k < max_path; ++k) pth[k] = -1;
+        n_acc[b] = 0;
+        bonus[b] = -1;
+        if (!oracle_tree_is_valid(par, n_nodes)) {
+            status[b] = ORACLE_BAD_TREE;
+            continue;
+        }
+        status[b] = ORACLE_OK;
+        int best_len = 0, best_end = -1;
+        for (int e = 0; e < n_nodes; ++e) {
+            int len = 0, ok = 1;
+            for (int u = e; u >= 0; u = par[u]) {
+                ++len;
+                if (par[u] >= 0 && tk[u] != tg[par[u]]) ok = 0;
+            }
+            if (ok && len <= max_path && len > best_len) {
+                best_len = len;
+                best_end = e;
+            }
+        }
+        if (best_end < 0) continue; /* only when max_path < 1 */
+        n_acc[b] = best_len;
+        bonus[b] = tg[best_end];
+        int k = best_len - 1;
+        for (int u = best_end; u >= 0; u = par[u]) pth[k--] = u;
+    }
+}
+
+/*
+ * Sec. 4.3 / Algorithm 4 in per-step form: the K/V rows of the accepted nodes
+ * are appended, in path order and without gaps, at logical positions
+ * L_b .. L_b + n_acc - 1 of sequence b; the physical slot of position p is
+ * page_table[b][p / P] * P + p % P.  A sequence whose pages cannot hold the
+ * new positions, or that would write below the shared prefix, gets
+ * ORACLE_CAPACITY and is left untouched.  slots is padded with -1.
+ */
+void oracle_kv_commit(uint16_t *k_pool, uint16_t *v_pool, int num_pages, int page_size,
+                      int n_kv_heads, int head_dim, const int32_t *page_table, int max_pages,
+                      int32_t *seq_lens, int shared_prefix_len,
+                      const uint16_t *k_tree, const uint16_t *v_tree, int batch, int n_nodes,
+                      const int32_t *path, const int32_t *n_acc, int max_path,
+                      int update_seq_lens, int32_t *slots, int32_t *status)
+{
+    const int D = head_dim;
+    for (int b = 0; b < batch; ++b) {
+        int32_t *sl = slots + (size_t)b * max_path;
+        for (int k = 0; k < max_path; ++k) sl[k] = -1;
+        const int L = seq_lens[b];
+        const int n = n_acc[b];
+        status[b] = ORACLE_OK;
+        if (n <= 0) continue;
+        int ok = (n <= max_path) && L >= 0 && L >= shared_prefix_len &&
+                 ((int64_t)L + n <= (int64_t)max_pages * page_size);
+        for (int k = 0; ok && k < n; ++k) {
+            const int32_t pg = page_table[(size_t)b * max_pages + (L + k) / page_size];
+            const int32_t node = path[(size_t)b * max_path + k];
+            if (pg < 0 || pg >= num_pages || node < 0 || node >= n_nodes) ok = 0;
+        }
+        if (!ok) {
+            status[b] = ORACLE_CAPACITY;
+            continue;
+        }
+        for (int k = 0; k < n; ++k) {
+            const int pos = L + k;
+            const int32_t pg = page_table[(size_t)b * max_pages + pos / page_size];
+            const int32_t node = path[(size_t)b * max_path + k];
+            sl[k] = pg * page_size + pos % page_size;
+            for (int h = 0; h < n_kv_heads; ++h) {
+                const size_t dst = (((size_t)pg * n_kv_heads + h) * page_size + pos % page_size) * D;
+                const size_t src = (((size_t)b * n_nodes + node) * n_kv_heads + h) * D;
+                memcpy(k_pool + dst, k_tree + src, sizeof(uint16_t) * D);
+                memcpy(v_pool + dst, v_tree + src, sizeof(uint16_t) * D);
+            }
+        }
+        if (update_seq_lens) seq_lens[b] = L + n;
+    }
+}
