@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of one batched tree-verification step (tree attention, acceptance, KV commit).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic batch: reader_verify_attn (ancestor masks
+encoded inside the call), reader_accept on the target logits, reader_kv_commit.  `value` is
+verified tree-tokens per second (batch * tree nodes / step time) with every input resident in
+HBM; `e2e` is the same with the step's inputs (Q, tree K/V, parent arrays, node tokens, logits)
+copied from pinned host memory and the results copied back inside the timed region.  Sequences are
+independent, so N GPUs run N replicas of the batch with no data-path collective (weak scaling).
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified tree-tokens/s (verify attention + acceptance + KV commit, 1 step)"
+UNIT = "tokens/s"
+LAUNCHES_PER_STEP = 6   # prepare, attention, combine, argmax, accept walk, commit
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.06] or [l for (_, l) in self.lines[-3:]]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def workload_config(w, name):
+    import numpy as np
+    return {"workload": name, "batch": int(w.batch), "tree_nodes": int(w.n_nodes), "n_q_heads": int(w.n_q_heads),
+            "n_kv_heads": int(w.n_kv_heads), "head_dim": int(w.head_dim), "page_size": int(w.page_size),
+            "committed_tokens": int(np.sum(w.seq_lens)), "shared_prefix_len": int(w.shared_prefix_len),
+            "vocab": int(w.vocab), "l2": "no flush: per-step inputs exceed the 126 MB L2"
+            if w.attn_algorithmic_bytes() + w.logits_bytes() > 2 * 126e6 else "fits L2: numbers are warm-cache"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU baseline: the checker as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+def cpu_sample_step(w, seqs):
+    """Runs the CPU checker on the given sequences of the workload (whole step); returns seconds."""
+    import copy
+    import numpy as np
+    import oracle
+    t0 = time.perf_counter()
+    for b in seqs:
+        s = copy.copy(w)
+        s.batch = 1
+        for f in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits"):
+            setattr(s, f, getattr(w, f)[b:b + 1])
+        s.page_table, s.seq_lens = w.page_table[b:b + 1], w.seq_lens[b:b + 1]
+        oracle.verify_attn(s.q, s.k_tree, s.v_tree, w.k_pool, w.v_pool, s.page_table, s.seq_lens, s.parent, w.scale)
+        tgt = oracle.argmax(s.logits)
+        a = oracle.accept(s.parent, s.node_tokens, tgt, w.max_path)
+        # commit on the sequence's own pages only (the checker copies the pool it is given)
+        used = s.page_table[0][s.page_table[0] >= 0]
+        remap = np.full(w.num_pages, -1, np.int32)
+        remap[used] = np.arange(len(used), dtype=np.int32)
+        pt = np.where(s.page_table >= 0, remap[np.maximum(s.page_table, 0)], -1).astype(np.int32)
+        oracle.kv_commit(w.k_pool[used], w.v_pool[used], pt, s.seq_lens, 0, s.k_tree, s.v_tree, a["path"], a["n_acc"])
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, budget_s=12.0):
+    import oracle
+    cores = oracle.num_threads()
+    done, spent = 0, 0.0
+    while done < w.batch and spent < budget_s:
+        spent += cpu_sample_step(w, [done])
+        done += 1
+    return {"value": done * w.n_nodes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"whole step on the first {done} of {w.batch} sequences ({done * w.n_nodes} tree tokens), "
+                      f"{spent:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2508_09072_b200 import workloads as W
+    oracle.build()
+    w = W.make(args.workload)
+    t1 = cpu_sample_step(w, [0])                      # also warms the page cache and the library
+    per_step = 120.0 / (args.steps + args.warmup)     # the whole run should end within a few minutes
+    n_seq = int(min(w.batch, max(1, per_step / max(t1, 1e-4))))
+    seqs = list(range(n_seq))
+    for _ in range(args.warmup):
+        cpu_sample_step(w, seqs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        cpu_sample_step(w, seqs)
+    dt = time.perf_counter() - t0
+    value = args.steps * n_seq * w.n_nodes / dt
+    cores = oracle.num_threads()
+    sample = f"each step = whole path on the first {n_seq} of {w.batch} sequences of {args.workload}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args.workload),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2508_09072_b200 import binding, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    peaks, peak_kind = load_peaks()
+
+    w = W.make(args.workload, seed_offset=rank)
+    rd = binding.Reader(local)
+    if args.kernel:
+        rd.set_attn_kernel(args.kernel)
+    d = binding.to_device(w, dev)
+    B, T = w.batch, w.n_nodes
+    seq_lens0 = d.cache.seq_lens.clone()
+    out = torch.empty_like(d.q)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    tgt = torch.empty((B, T), dtype=torch.int32, device=dev)
+    acc_out = (torch.empty((B, w.max_path), dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+               torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev))
+    slots = torch.empty((B, w.max_path), dtype=torch.int32, device=dev)
+    cstat = torch.empty(B, dtype=torch.int32, device=dev)
+    ws = rd.workspace(B, T, w.n_q_heads, w.n_kv_heads, w.head_dim)
+
+    def step(ev=None):
+        d.cache.seq_lens.copy_(seq_lens0)            # harness: rewind the cache length
+        if ev:
+            ev[0].record()
+        rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=out, status=status, workspace=ws)
+        if ev:
+            ev[1].record()
+        rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=tgt, workspace=ws, outs=acc_out)
+        if ev:
+            ev[2].record()
+        rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc_out[0], acc_out[1], slots=slots, status=cstat)
+        if ev:
+            ev[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def mk():
+        return torch.cuda.Event(enable_timing=True)
+
+    # ---- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        step()
+    K = args.steps
+    evs = [[mk() for _ in range(4)] for _ in range(K)]
+    kev = [(mk(), mk()) for _ in range(K)]
+    for a, b in kev:                                  # create the handles
+        a.record(); b.record()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_wall0 = time.time()
+    e0, e1 = mk(), mk()
+    e0.record()
+    for i in range(K):
+        rd.set_timing_events(*kev[i])
+        step(evs[i])
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    rd.set_timing_events(None, None)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / K
+    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / K
+    t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / K
+    t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / K
+    assert int(status.max().item()) == 0 and int(cstat.max().item()) == 0 and int(acc_out[3].max().item()) == 0
+
+    # ---- end to end: host buffers in, results out, every step
+    host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits")}
+    host_out = {"out": torch.empty(out.shape, dtype=out.dtype).pin_memory(),
+                "path": torch.empty(acc_out[0].shape, dtype=torch.int32).pin_memory(),
+                "n_acc": torch.empty(B, dtype=torch.int32).pin_memory(),
+                "bonus": torch.empty(B, dtype=torch.int32).pin_memory(),
+                "slots": torch.empty(slots.shape, dtype=torch.int32).pin_memory()}
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_step():
+        for k, t in host_in.items():
+            getattr(d, k).copy_(t, non_blocking=True)
+        step()
+        host_out["out"].copy_(out, non_blocking=True)
+        host_out["path"].copy_(acc_out[0], non_blocking=True)
+        host_out["n_acc"].copy_(acc_out[1], non_blocking=True)
+        host_out["bonus"].copy_(acc_out[2], non_blocking=True)
+        host_out["slots"].copy_(slots, non_blocking=True)
+        torch.cuda.current_stream().synchronize()     # the caller needs the result before the next step
+
+    Ke = max(3, min(K, args.e2e_steps))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    f0, f1 = mk(), mk()
+    f0.record()
+    for _ in range(Ke):
+        e2e_step()
+    f1.record()
+    barrier()
+    ms_e2e = f0.elapsed_time(f1)
+
+    # ---- max over ranks
+    t = torch.tensor([ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel = t.tolist()
+
+    if rank == 0:
+        tokens = B * T * world
+        value = tokens * K / (ms_total * 1e-3)
+        e2e = tokens * Ke / (ms_e2e * 1e-3)
+        attn_bytes = w.attn_algorithmic_bytes()
+        attn_flops = w.attn_algorithmic_flops()
+        kernels = {
+            "verify_attn": {"ms": t_attn_kernel, "call_ms": t_attn_call, "algorithmic_bytes": attn_bytes,
+                            "gbs": attn_bytes / (t_attn_kernel * 1e-3) / 1e9,
+                            "algorithmic_flops": attn_flops, "tflops": attn_flops / (t_attn_kernel * 1e-3) / 1e12},
+            "accept": {"call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
+                       "gbs": w.logits_bytes() / (t_accept * 1e-3) / 1e9},
+            "kv_commit": {"call_ms": t_commit},
+        }
+        t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_tc = attn_flops / (peaks["bf16_tflops_sustained"] * 1e12)
+        kernels["verify_attn"]["binding_bound"] = "hbm" if t_hbm >= t_tc else "tensor"
+        kernels["verify_attn"]["binding_frac"] = max(t_hbm, t_tc) / (t_attn_kernel * 1e-3)
+        if t_attn_kernel >= t_accept:
+            a = kernels["verify_attn"]["gbs"]
+            roof = {"kernel": "verify_attn", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind}
+        else:
+            a = kernels["accept"]["gbs"]
+            roof = {"kernel": "accept (target argmax)", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args.workload),
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke},
+            "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "kernels": kernels,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    rd.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--kernel", type=int, default=0, help="attention kernel: 0 auto, 1 CUDA-core, 2 tensor-core")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

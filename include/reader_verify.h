@@ -1,0 +1,184 @@
+/*
+ * reader_verify.h -- C ABI of the batched tree-verification step of READER-style lossless
+ * speculative decoding, implemented as hand-written CUDA for sm_100a (NVIDIA B200).
+ *
+ * One decoding step of the method (Algorithm 1, lines 15-16 and 18-20) hands a draft tree per
+ * sequence to the target model, which scores every node in one pass (Sec. 3.2), keeps the
+ * longest root path the model agrees with (Algorithm 5; Appendix C, invariants 1-3) and appends
+ * the accepted entries to the KV cache without gaps (Sec. 4.3, Algorithm 4).  This library is
+ * the attention, acceptance and cache part of that step:
+ *
+ *     reader_tree_encode   parent array  ->  per-node ancestor bitmask           (Sec. 3.2 mask)
+ *     reader_verify_attn   tree-masked attention over paged cache + tree K/V     (Sec. 3.2)
+ *     reader_accept        target argmax + longest consistent root path          (Algorithm 5)
+ *     reader_kv_commit     accepted K/V rows -> cache tail, seq_lens += n_acc    (Algorithm 4)
+ *
+ * Conventions common to every call
+ *   - Every pointer named below is a DEVICE pointer owned by the caller unless it says "host".
+ *     The library allocates no device memory; scratch comes from the caller's workspace.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it: none of them
+ *     synchronises or reads device data on the host.
+ *   - Tensors are dense, row-major, last index fastest.  bf16 tensors are raw 16-bit patterns.
+ *     Pointers to bf16/f32/u64 tensors must be 16-byte aligned.
+ *   - Errors have two channels.  (1) The return value reports what the host can check (null or
+ *     misaligned pointers, unsupported shapes, workspace too small, a CUDA launch error); on
+ *     such an error nothing has been launched.  (2) `status_out[b]` (device, one word per
+ *     sequence) reports what only the data can tell: a malformed parent array, a page id
+ *     outside the pool, a length beyond the page table.  A sequence with a non-zero status gets
+ *     defined outputs (attention rows and lse zero; n_acc 0, path -1, bonus -1; nothing
+ *     committed) and does not disturb the others.  No kernel traps, asserts or waits unbounded.
+ *   - Tree convention: node 0 is the root = the last token already chosen by the target model
+ *     (its K/V is part of the tree tensors, not yet of the cache); parent[0] = -1 and
+ *     0 <= parent[j] < j.  At most READER_MAX_NODES nodes.
+ */
+#ifndef READER_VERIFY_H
+#define READER_VERIFY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define READER_MAX_NODES 128
+#define READER_PAGE_SIZE 64
+
+typedef struct reader_ctx reader_ctx; /* opaque: device id, SM count, driver entry points */
+
+typedef enum {
+    READER_OK = 0,
+    READER_ERR_INVALID_ARG = 1, /* null/misaligned pointer, size out of range */
+    READER_ERR_BAD_TREE = 2,    /* status word: parent array breaks the tree convention */
+    READER_ERR_CAPACITY = 3,    /* status word: length beyond the page table / commit has no room */
+    READER_ERR_WORKSPACE = 4,   /* workspace smaller than reader_workspace_bytes() */
+    READER_ERR_UNSUPPORTED = 5, /* shape the kernels are not built for */
+    READER_ERR_TIMEOUT = 6,     /* status word: a bounded device-side wait gave up */
+    READER_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed */
+    READER_ERR_BAD_PAGE = 8     /* status word: page-table entry outside [0, num_pages) */
+} reader_status;
+
+/*
+ * One layer's paged KV cache (Sec. 4.3: per-sample cache without internal padding).
+ *   k_pool, v_pool   bf16 [num_pages][n_kv_heads][page_size][head_dim]
+ *   page_table       i32  [batch][max_pages_per_seq]; entry p of row b is the pool page that
+ *                    holds logical positions p*page_size .. p*page_size+page_size-1 of sequence b
+ *   seq_lens         i32  [batch] committed tokens per sequence; read by reader_verify_attn,
+ *                    updated by reader_kv_commit
+ *   shared_prefix_len  tokens (multiple of page_size, 0 = none) whose pages are the same pool
+ *                    pages in every row of page_table (stored once); commits never write there
+ * page_size must be READER_PAGE_SIZE; head_dim 64 or 128.
+ */
+typedef struct {
+    void *k_pool;
+    void *v_pool;
+    int32_t num_pages, page_size, n_kv_heads, head_dim;
+    const int32_t *page_table;
+    int32_t max_pages_per_seq;
+    int32_t *seq_lens;
+    int32_t shared_prefix_len;
+} reader_kv_cache;
+
+/*
+ * The draft trees of one step (Sec. 3.2; built by the drafting side of Algorithm 1).
+ *   parent     i32 [batch][n_nodes]
+ *   anc_mask   u64 [batch][n_nodes][2]  bit i of the 128-bit word of node j is set iff node i is
+ *              j itself or an ancestor of j (from reader_tree_encode); NULL = encode internally
+ */
+typedef struct {
+    int32_t batch, n_nodes;
+    const int32_t *parent;
+    const uint64_t *anc_mask;
+} reader_tree;
+
+/* Creates a context for CUDA device `device` (host call; may initialise the CUDA context).
+ * *out is host memory owned by the library until reader_destroy. */
+reader_status reader_create(reader_ctx **out, int device);
+void reader_destroy(reader_ctx *ctx);
+const char *reader_status_string(reader_status s);
+
+/* Chooses the attention kernel: 0 = automatic (tensor-core kernel where the shape allows, else
+ * the CUDA-core kernel), 1 = always the CUDA-core kernel, 2 = tensor-core kernel or
+ * READER_ERR_UNSUPPORTED.  Both compute Sec. 3.2's attention; this is a testing aid. Host call. */
+reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
+
+/* Profiling aid (host call): when both are non-NULL cudaEvent_t handles, the next calls of
+ * reader_verify_attn record `start` on the stream right before the main attention kernel and
+ * `stop` right after it (the preparation and combine kernels lie outside).  NULL, NULL turns it off. */
+reader_status reader_set_timing_events(reader_ctx *ctx, void *start, void *stop);
+
+/* Bytes of device scratch that reader_verify_attn / reader_accept need for at most `max_batch`
+ * sequences of at most `max_nodes` nodes.  Host call, no CUDA work.  Returns 0 on bad arguments. */
+size_t reader_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes,
+                              int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim);
+
+/*
+ * Sec. 3.2 decoding mask.  For every sequence b and node j writes the 128-bit ancestor-or-self
+ * set anc_mask_out[b][j][0..1] and level_out[b][j] = number of nodes on the path root..j (nullable).
+ * status_out[b] = READER_ERR_BAD_TREE when parent[b] breaks the tree convention (its masks are
+ * then zero).  1 <= n_nodes <= READER_MAX_NODES.
+ */
+reader_status reader_tree_encode(reader_ctx *ctx, const int32_t *parent, int32_t batch, int32_t n_nodes,
+                                 uint64_t *anc_mask_out, int32_t *level_out, int32_t *status_out,
+                                 void *stream);
+
+/*
+ * Sec. 3.2 verification attention.  For sequence b, node j and query head h (KV head h / G,
+ * G = n_q_heads / n_kv_heads) the query q[b][j][h] attends, with scores scaled by
+ * softmax_scale, to the committed keys 0 .. seq_lens[b]-1 of the paged cache and to the tree
+ * keys k_tree[b][i] of the nodes i that are j or an ancestor of j.
+ *   q, out          bf16 [batch][n_nodes][n_q_heads][head_dim]
+ *   k_tree, v_tree  bf16 [batch][n_nodes][n_kv_heads][head_dim]
+ *   lse_out         f32  [batch][n_nodes][n_q_heads], natural log of the softmax denominator; nullable
+ *   workspace       at least reader_workspace_bytes(...) bytes, 256-byte aligned; contents are
+ *                   scratch, calls that share it must not overlap on the GPU
+ *   status_out      i32 [batch]
+ * Arithmetic: bf16 inputs, fp32 accumulation and softmax, probabilities rounded to bf16 before the
+ * value product where tensor cores are used, bf16 (nearest-even) output.
+ */
+reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_heads,
+                                 const void *k_tree, const void *v_tree,
+                                 const reader_kv_cache *cache, const reader_tree *tree,
+                                 float softmax_scale, void *out, float *lse_out,
+                                 void *workspace, size_t workspace_bytes, int32_t *status_out,
+                                 void *stream);
+
+/*
+ * Algorithm 5 step 2 with the greedy policy of Appendix C.  If `logits` (f32
+ * [batch][n_nodes][vocab]) is given, target_ids[b][j] is first set to the lowest index of the
+ * row maximum (a NaN never wins; a NaN in slot 0 counts as -inf); otherwise target_ids is read
+ * as given (any policy's per-node choice, e.g. a sampler driven by coupled uniforms).
+ * A node is accepted when it is the root or its parent is accepted and
+ * node_tokens[node] == target_ids[parent].  Returns the longest accepted root path with at most
+ * max_path nodes (lowest end node among equals; equal sibling tokens are all followed):
+ *   path_out   i32 [batch][max_path] node ids from the root, padded with -1
+ *   n_acc_out  i32 [batch] nodes on the path, root counted (>= 1 for a valid tree)
+ *   bonus_out  i32 [batch] target_ids at the end node: the token to emit after the path
+ * The tokens appended to the output this step are node_tokens[path[1..n_acc-1]] then bonus.
+ * workspace: as for reader_verify_attn (used only when logits is given).
+ */
+reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens,
+                            const float *logits, int32_t vocab, int32_t *target_ids,
+                            int32_t max_path, int32_t *path_out, int32_t *n_acc_out,
+                            int32_t *bonus_out, void *workspace, size_t workspace_bytes,
+                            int32_t *status_out, void *stream);
+
+/*
+ * Sec. 4.3 / Algorithm 4 in per-step form.  For k < n_acc[b] the K/V rows of node path[b][k]
+ * (all KV heads) are copied to logical position seq_lens[b] + k of sequence b, i.e. pool slot
+ * page_table[b][(L+k)/page_size]*page_size + (L+k)%page_size, which is also written to
+ * slots_out[b][k] (i32 [batch][max_path], -1 padded).  If update_seq_lens != 0, seq_lens[b] +=
+ * n_acc[b] afterwards (pass 0 for all but the last layer that shares seq_lens).  A sequence
+ * whose page table cannot hold the new positions, or that would write below
+ * shared_prefix_len, gets READER_ERR_CAPACITY and is left untouched.
+ */
+reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const void *k_tree,
+                               const void *v_tree, int32_t batch, int32_t n_nodes,
+                               const int32_t *path, const int32_t *n_acc, int32_t max_path,
+                               int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out,
+                               void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* READER_VERIFY_H */

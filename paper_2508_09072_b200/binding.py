@@ -1,0 +1,291 @@
+"""ctypes binding of ``libreader_verify.so``: argument marshalling only.
+
+Every step of the verification path runs in the library's CUDA kernels.  PyTorch is used for
+device memory and streams; tensors are passed as raw device pointers.  bf16 tensors are
+``torch.bfloat16``.  There is no CPU fallback: if the library is missing or no CUDA device is
+present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_float, c_int32, c_size_t, c_void_p
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libreader_verify.so")
+
+OK, ERR_INVALID_ARG, ERR_BAD_TREE, ERR_CAPACITY, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_CUDA, ERR_BAD_PAGE = range(9)
+
+EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
+           "reader_set_timing_events",
+           "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
+           "reader_kv_commit")
+
+
+class ReaderError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class _KvCache(Structure):
+    _fields_ = [("k_pool", c_void_p), ("v_pool", c_void_p), ("num_pages", c_int32), ("page_size", c_int32),
+                ("n_kv_heads", c_int32), ("head_dim", c_int32), ("page_table", c_void_p),
+                ("max_pages_per_seq", c_int32), ("seq_lens", c_void_p), ("shared_prefix_len", c_int32)]
+
+
+class _Tree(Structure):
+    _fields_ = [("batch", c_int32), ("n_nodes", c_int32), ("parent", c_void_p), ("anc_mask", c_void_p)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the shared library (no CUDA call is made by loading it)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2508_09072_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.reader_create.argtypes = [POINTER(c_void_p), c_int32]
+    lib.reader_create.restype = c_int32
+    lib.reader_destroy.argtypes = [c_void_p]
+    lib.reader_destroy.restype = None
+    lib.reader_status_string.argtypes = [c_int32]
+    lib.reader_status_string.restype = ctypes.c_char_p
+    lib.reader_set_attn_kernel.argtypes = [c_void_p, c_int32]
+    lib.reader_set_attn_kernel.restype = c_int32
+    lib.reader_set_timing_events.argtypes = [c_void_p, c_void_p, c_void_p]
+    lib.reader_set_timing_events.restype = c_int32
+    lib.reader_workspace_bytes.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32]
+    lib.reader_workspace_bytes.restype = c_size_t
+    lib.reader_tree_encode.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.reader_tree_encode.restype = c_int32
+    lib.reader_verify_attn.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, POINTER(_KvCache),
+                                       POINTER(_Tree), c_float, c_void_p, c_void_p, c_void_p, c_size_t,
+                                       c_void_p, c_void_p]
+    lib.reader_verify_attn.restype = c_int32
+    lib.reader_accept.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
+                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.reader_accept.restype = c_int32
+    lib.reader_kv_commit.argtypes = [c_void_p, POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
+                                     c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
+    lib.reader_kv_commit.restype = c_int32
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().reader_status_string(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: need a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+@dataclass
+class KvCache:
+    """One layer's paged cache; tensors live on the device and are owned by the caller."""
+    k_pool: torch.Tensor      # bf16 [num_pages, Hkv, page_size, D]
+    v_pool: torch.Tensor
+    page_table: torch.Tensor  # i32 [B, max_pages]
+    seq_lens: torch.Tensor    # i32 [B]
+    shared_prefix_len: int = 0
+
+    def _c(self) -> _KvCache:
+        _dev(self.k_pool, torch.bfloat16, "k_pool"); _dev(self.v_pool, torch.bfloat16, "v_pool")
+        _dev(self.page_table, torch.int32, "page_table"); _dev(self.seq_lens, torch.int32, "seq_lens")
+        n, h, p, d = self.k_pool.shape
+        return _KvCache(self.k_pool.data_ptr(), self.v_pool.data_ptr(), n, p, h, d, self.page_table.data_ptr(),
+                        self.page_table.shape[1], self.seq_lens.data_ptr(), int(self.shared_prefix_len))
+
+
+class Reader:
+    """Handle on the library for one CUDA device (wraps reader_create / reader_destroy)."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2508_09072_b200 needs a CUDA device; there is no CPU fallback")
+        self.lib = load_library()
+        self.device = int(device)
+        torch.cuda.set_device(self.device)
+        torch.zeros(1, device=f"cuda:{self.device}")   # make sure the context exists
+        h = c_void_p()
+        st = self.lib.reader_create(ctypes.byref(h), self.device)
+        if st != OK:
+            raise ReaderError(st, "reader_create")
+        self._h = h
+        self._ws: Optional[torch.Tensor] = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.reader_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- helpers
+    def set_attn_kernel(self, which: int) -> None:
+        st = self.lib.reader_set_attn_kernel(self._h, int(which))
+        if st != OK:
+            raise ReaderError(st, "reader_set_attn_kernel")
+
+    def set_timing_events(self, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+        """Events (created with enable_timing=True and already recorded once, so that their handles
+        exist) that reader_verify_attn records around its main kernel; None, None turns it off."""
+        a = None if start is None else c_void_p(start.cuda_event)
+        b = None if stop is None else c_void_p(stop.cuda_event)
+        st = self.lib.reader_set_timing_events(self._h, a, b)
+        if st != OK:
+            raise ReaderError(st, "reader_set_timing_events")
+
+    def workspace_bytes(self, max_batch: int, max_nodes: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
+        return int(self.lib.reader_workspace_bytes(self._h, max_batch, max_nodes, n_q_heads, n_kv_heads, head_dim))
+
+    def workspace(self, max_batch: int, max_nodes: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> torch.Tensor:
+        """A cached device buffer large enough for the given limits (torch allocation)."""
+        need = self.workspace_bytes(max_batch, max_nodes, n_q_heads, n_kv_heads, head_dim)
+        if need == 0:
+            raise ReaderError(ERR_INVALID_ARG, "reader_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
+        return self._ws
+
+    # ---- the calls
+    def tree_encode(self, parent: torch.Tensor, anc_mask: Optional[torch.Tensor] = None,
+                    level: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+        _dev(parent, torch.int32, "parent")
+        B, T = parent.shape
+        dev = parent.device
+        anc_mask = anc_mask if anc_mask is not None else torch.empty((B, T, 2), dtype=torch.int64, device=dev)
+        level = level if level is not None else torch.empty((B, T), dtype=torch.int32, device=dev)
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=dev)
+        st = self.lib.reader_tree_encode(self._h, _ptr(parent), B, T, _ptr(anc_mask), _ptr(level), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_tree_encode")
+        return anc_mask, level, status
+
+    def verify_attn(self, q: torch.Tensor, k_tree: torch.Tensor, v_tree: torch.Tensor, cache: KvCache,
+                    parent: torch.Tensor, scale: float, anc_mask: Optional[torch.Tensor] = None,
+                    out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                    status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+        _dev(q, torch.bfloat16, "q"); _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        _dev(parent, torch.int32, "parent")
+        B, T, Hq, D = q.shape
+        Hkv = k_tree.shape[2]
+        out = out if out is not None else torch.empty_like(q)
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=q.device)
+        ws = workspace if workspace is not None else self.workspace(max(B, 1), T, Hq, Hkv, D)
+        tree = _Tree(B, T, parent.data_ptr(), None if anc_mask is None else anc_mask.data_ptr())
+        c = cache._c()
+        st = self.lib.reader_verify_attn(self._h, _ptr(q), Hq, _ptr(k_tree), _ptr(v_tree), ctypes.byref(c),
+                                         ctypes.byref(tree), float(scale), _ptr(out), _ptr(lse), _ptr(ws),
+                                         ws.numel(), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_verify_attn")
+        return out, status
+
+    def accept(self, parent: torch.Tensor, node_tokens: torch.Tensor, max_path: int,
+               logits: Optional[torch.Tensor] = None, target_ids: Optional[torch.Tensor] = None,
+               workspace: Optional[torch.Tensor] = None, outs=None):
+        _dev(parent, torch.int32, "parent"); _dev(node_tokens, torch.int32, "node_tokens")
+        B, T = parent.shape
+        dev = parent.device
+        vocab = 0
+        if logits is not None:
+            _dev(logits, torch.float32, "logits")
+            vocab = logits.shape[-1]
+            if target_ids is None:
+                target_ids = torch.empty((B, T), dtype=torch.int32, device=dev)
+        elif target_ids is None:
+            raise TypeError("accept: give logits or target_ids")
+        _dev(target_ids, torch.int32, "target_ids")
+        if outs is None:
+            outs = (torch.empty((B, max_path), dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev))
+        path, n_acc, bonus, status = outs
+        ws = workspace if workspace is not None else self.workspace(max(B, 1), T, 1, 1, 64)
+        tree = _Tree(B, T, parent.data_ptr(), None)
+        st = self.lib.reader_accept(self._h, ctypes.byref(tree), _ptr(node_tokens), _ptr(logits), vocab,
+                                    _ptr(target_ids), int(max_path), _ptr(path), _ptr(n_acc), _ptr(bonus),
+                                    _ptr(ws), ws.numel(), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_accept")
+        return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
+
+    def kv_commit(self, cache: KvCache, k_tree: torch.Tensor, v_tree: torch.Tensor, path: torch.Tensor,
+                  n_acc: torch.Tensor, update_seq_lens: bool = True, slots: Optional[torch.Tensor] = None,
+                  status: Optional[torch.Tensor] = None):
+        _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        _dev(path, torch.int32, "path"); _dev(n_acc, torch.int32, "n_acc")
+        B, T = k_tree.shape[:2]
+        max_path = path.shape[1]
+        slots = slots if slots is not None else torch.empty((B, max_path), dtype=torch.int32, device=path.device)
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=path.device)
+        c = cache._c()
+        st = self.lib.reader_kv_commit(self._h, ctypes.byref(c), _ptr(k_tree), _ptr(v_tree), B, T, _ptr(path),
+                                       _ptr(n_acc), max_path, int(bool(update_seq_lens)), _ptr(slots), _ptr(status),
+                                       _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_kv_commit")
+        return slots, status
+
+
+# ---------------------------------------------------------------------------------------------
+# moving a host workload onto the device (no arithmetic)
+# ---------------------------------------------------------------------------------------------
+def bf16_tensor(bits, device) -> torch.Tensor:
+    """numpy uint16 bit patterns -> torch.bfloat16 tensor on `device` (reinterpretation, no rounding)."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)
+
+
+def bf16_bits(t: torch.Tensor):
+    """torch.bfloat16 tensor -> numpy uint16 bit patterns on the host."""
+    import numpy as np
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@dataclass
+class DeviceWorkload:
+    q: torch.Tensor
+    k_tree: torch.Tensor
+    v_tree: torch.Tensor
+    cache: KvCache
+    parent: torch.Tensor
+    node_tokens: torch.Tensor
+    logits: Optional[torch.Tensor]
+    scale: float
+    max_path: int
+
+
+def to_device(w, device="cuda:0", with_logits: bool = True) -> DeviceWorkload:
+    cache = KvCache(bf16_tensor(w.k_pool, device), bf16_tensor(w.v_pool, device),
+                    torch.from_numpy(w.page_table).to(device), torch.from_numpy(w.seq_lens).to(device),
+                    w.shared_prefix_len)
+    logits = torch.from_numpy(w.logits).to(device) if (with_logits and w.logits is not None) else None
+    return DeviceWorkload(bf16_tensor(w.q, device), bf16_tensor(w.k_tree, device), bf16_tensor(w.v_tree, device),
+                          cache, torch.from_numpy(w.parent).to(device), torch.from_numpy(w.node_tokens).to(device),
+                          logits, float(w.scale), int(w.max_path))

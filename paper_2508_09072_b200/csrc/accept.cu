@@ -1,0 +1,182 @@
+// Acceptance (Algorithm 5 step 2; Appendix C invariants 2-3 with the greedy policy): row argmax
+// of the target logits with a lowest-index tie-break, then the longest root path whose every
+// non-root node carries the token the target model picks after its parent.
+#include <limits.h>
+
+#include "common.cuh"
+#include "tree.cuh"
+
+namespace reader {
+
+struct Best {
+    float v;
+    int i;
+};
+
+__device__ __forceinline__ Best better(Best a, Best b) {
+    // larger value wins; equal values: lower index.  NaNs never enter (they fail every '>' below).
+    if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
+    return a;
+}
+
+// grid (rows, splits): block (r, s) scans columns [s*chunk, min(V, (s+1)*chunk)) of row r.
+template <bool kVec>
+__global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ logits, int64_t vocab, int chunk,
+                                                     int splits, float *__restrict__ part_val,
+                                                     int32_t *__restrict__ part_idx) {
+    const int64_t row = blockIdx.x;
+    const int split = blockIdx.y;
+    const int c0 = split * chunk;
+    const int c1 = (int)min((int64_t)c0 + chunk, vocab);
+    const float *src = logits + row * vocab;
+    Best best{-INFINITY, INT_MAX};
+    if (kVec) {
+        const float4 *v4 = reinterpret_cast<const float4 *>(src + c0);
+        const int n4 = (c1 - c0) >> 2;
+        int i = threadIdx.x;
+        for (; i + 3 * 256 < n4; i += 4 * 256) {
+            float4 a[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a[u] = __ldcs(v4 + i + u * 256);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int at = c0 + 4 * (i + u * 256);
+                if (a[u].x > best.v) { best.v = a[u].x; best.i = at; }
+                if (a[u].y > best.v) { best.v = a[u].y; best.i = at + 1; }
+                if (a[u].z > best.v) { best.v = a[u].z; best.i = at + 2; }
+                if (a[u].w > best.v) { best.v = a[u].w; best.i = at + 3; }
+            }
+        }
+        for (; i < n4; i += 256) {
+            const float4 a = __ldcs(v4 + i);
+            const int at = c0 + 4 * i;
+            if (a.x > best.v) { best.v = a.x; best.i = at; }
+            if (a.y > best.v) { best.v = a.y; best.i = at + 1; }
+            if (a.z > best.v) { best.v = a.z; best.i = at + 2; }
+            if (a.w > best.v) { best.v = a.w; best.i = at + 3; }
+        }
+        for (int c = c0 + 4 * n4 + threadIdx.x; c < c1; c += 256) {
+            const float a = src[c];
+            if (a > best.v) { best.v = a; best.i = c; }
+        }
+    } else {
+        for (int c = c0 + threadIdx.x; c < c1; c += 256) {
+            const float a = src[c];
+            if (a > best.v) { best.v = a; best.i = c; }
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        Best o{__shfl_xor_sync(0xffffffffu, best.v, d), __shfl_xor_sync(0xffffffffu, best.i, d)};
+        best = better(best, o);
+    }
+    __shared__ Best wb[8];
+    if ((threadIdx.x & 31) == 0) wb[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int k = 1; k < 8; ++k) best = better(best, wb[k]);
+        part_val[row * splits + split] = best.v;
+        part_idx[row * splits + split] = best.i;
+    }
+}
+
+void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits, float *part_val,
+                   int32_t *part_idx, cudaStream_t st) {
+    if (rows <= 0) return;
+    int chunk = (int)((vocab + splits - 1) / splits);
+    chunk = (chunk + 3) & ~3;
+    dim3 grid((unsigned)rows, (unsigned)splits);
+    if (vocab % 4 == 0)
+        argmax_kernel<true><<<grid, 256, 0, st>>>(logits, vocab, chunk, splits, part_val, part_idx);
+    else
+        argmax_kernel<false><<<grid, 256, 0, st>>>(logits, vocab, chunk, splits, part_val, part_idx);
+}
+
+// One warp per sequence.
+__global__ void __launch_bounds__(128) accept_kernel(const int32_t *__restrict__ parent,
+                                                     const int32_t *__restrict__ tok, int32_t *__restrict__ target,
+                                                     int B, int T, int max_path, const float *__restrict__ part_val,
+                                                     const int32_t *__restrict__ part_idx, int splits,
+                                                     int32_t *__restrict__ path, int32_t *__restrict__ n_acc,
+                                                     int32_t *__restrict__ bonus, int32_t *__restrict__ status) {
+    __shared__ int32_t par_s[4][kMaxNodes];
+    __shared__ int32_t tgt_s[4][kMaxNodes];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 4 + warp;
+    if (b >= B) return;
+    int32_t *par = par_s[warp], *tgt = tgt_s[warp];
+
+    for (int j = lane; j < T; j += 32) {
+        par[j] = parent[(size_t)b * T + j];
+        int t;
+        if (splits > 0) {
+            Best best{-INFINITY, INT_MAX};
+            const size_t row = (size_t)b * T + j;
+            for (int s = 0; s < splits; ++s) best = better(best, Best{part_val[row * splits + s], part_idx[row * splits + s]});
+            t = best.i == INT_MAX ? 0 : best.i;
+            target[row] = t;
+        } else {
+            t = target[(size_t)b * T + j];
+        }
+        tgt[j] = t;
+    }
+    __syncwarp();
+    const bool valid = warp_tree_valid(par, T, lane);
+    for (int k = lane; k < max_path; k += 32) path[(size_t)b * max_path + k] = -1;
+    if (!valid) {
+        if (lane == 0) { n_acc[b] = 0; bonus[b] = -1; status[b] = READER_ERR_BAD_TREE; }
+        return;
+    }
+    // which nodes carry the token the target model picks after their parent
+    uint32_t okw[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int j = lane + 32 * i;
+        const bool ok = j < T && (j == 0 || tok[(size_t)b * T + j] == tgt[par[j]]);
+        okw[i] = __ballot_sync(0xffffffffu, ok);
+    }
+    const uint64_t ok_lo = (uint64_t)okw[0] | ((uint64_t)okw[1] << 32);
+    const uint64_t ok_hi = (uint64_t)okw[2] | ((uint64_t)okw[3] << 32);
+
+    // a node is accepted iff it and all its ancestors are ok; deepest wins, lowest index among equals
+    int key = 0;
+    uint64_t my_lo[4], my_hi[4];
+    int my_lv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int j = lane + 32 * i;
+        my_lo[i] = my_hi[i] = 0; my_lv[i] = 0;
+        if (j < T) {
+            node_ancestors(par, T, j, my_lo[i], my_hi[i], my_lv[i]);
+            const bool acc = ((my_lo[i] & ~ok_lo) | (my_hi[i] & ~ok_hi)) == 0;
+            if (acc && my_lv[i] <= max_path) key = max(key, my_lv[i] * 256 + (255 - j));
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, d));
+    const int end = 255 - (key & 255);
+    const int n = key >> 8;
+    uint64_t e_lo = 0, e_hi = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if ((end >> 5) == i) {
+            e_lo = __shfl_sync(0xffffffffu, my_lo[i], end & 31);
+            e_hi = __shfl_sync(0xffffffffu, my_hi[i], end & 31);
+        }
+    __syncwarp();   // the -1 fill above is ordered before the path writes below
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int j = lane + 32 * i;
+        const bool on = j < 64 ? (e_lo >> j) & 1 : (e_hi >> (j - 64)) & 1;
+        if (j < T && on) path[(size_t)b * max_path + my_lv[i] - 1] = j;
+    }
+    if (lane == 0) { n_acc[b] = n; bonus[b] = tgt[end]; status[b] = READER_OK; }
+}
+
+void launch_accept(const int32_t *parent, const int32_t *tok, int32_t *target, int B, int T, int max_path,
+                   const float *part_val, const int32_t *part_idx, int splits, int32_t *path, int32_t *n_acc,
+                   int32_t *bonus, int32_t *status, cudaStream_t st) {
+    if (B <= 0) return;
+    accept_kernel<<<(B + 3) / 4, 128, 0, st>>>(parent, tok, target, B, T, max_path, part_val, part_idx, splits,
+                                               path, n_acc, bonus, status);
+}
+
+}  // namespace reader

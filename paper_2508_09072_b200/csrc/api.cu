@@ -1,0 +1,271 @@
+// C-ABI entry points: argument validation, workspace carving and kernel sequencing.
+// Nothing here touches device data from the host or synchronises the stream.
+#include <new>
+
+#include "common.cuh"
+#include "verify_attn_sm100.cuh"
+
+struct reader_ctx {
+    int device;
+    int n_sm;
+    int attn_kernel;  // 0 auto, 1 generic (CUDA cores), 2 tensor-core kernel only
+    reader::Sm100Host sm100;
+    cudaEvent_t ev_start, ev_stop;  // optional timing hooks around the main attention kernel
+};
+
+namespace {
+
+using namespace reader;
+
+constexpr int kMaxSplits = 64;
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct WsLayout {
+    size_t error_flag, seq_tile_start, seq_ntiles, seq_npages, anc, partial_ml, partial_o, amax_val, amax_idx, total;
+};
+
+inline int max_ctas(const reader_ctx *ctx) { return 2 * ctx->n_sm; }
+
+WsLayout ws_layout(const reader_ctx *ctx, int B, int T, int D) {
+    WsLayout w{};
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes); return o; };
+    const size_t slots = 2 * (size_t)max_ctas(ctx);
+    w.error_flag = take(sizeof(int32_t));
+    w.seq_tile_start = take(sizeof(int32_t) * ((size_t)B + 1));
+    w.seq_ntiles = take(sizeof(int32_t) * (size_t)B);
+    w.seq_npages = take(sizeof(int32_t) * (size_t)B);
+    w.anc = take(sizeof(uint64_t) * 2 * (size_t)B * T);
+    w.partial_ml = take(sizeof(float) * 2 * slots * kTileM);
+    w.partial_o = take(sizeof(float) * slots * kTileM * (size_t)D);
+    w.amax_val = take(sizeof(float) * (size_t)B * T * kMaxSplits);
+    w.amax_idx = take(sizeof(int32_t) * (size_t)B * T * kMaxSplits);
+    w.total = at;
+    return w;
+}
+
+inline bool shape_ok(int B, int T, int Hq, int Hkv, int D) {
+    return B >= 0 && T >= 1 && T <= kMaxNodes && Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && (D == 64 || D == 128);
+}
+
+inline reader_status check_device(const reader_ctx *ctx) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return READER_ERR_CUDA;
+    return dev == ctx->device ? READER_OK : READER_ERR_INVALID_ARG;
+}
+
+inline reader_status launch_status() { return cudaGetLastError() == cudaSuccess ? READER_OK : READER_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+reader_status reader_create(reader_ctx **out, int device) {
+    if (!out) return READER_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n_sm = 0, major = 0;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) {
+        cudaGetLastError();
+        return READER_ERR_CUDA;
+    }
+    if (major != 10) return READER_ERR_UNSUPPORTED;   // the kernels are sm_100a code only
+    reader_ctx *ctx = new (std::nothrow) reader_ctx();
+    if (!ctx) return READER_ERR_CUDA;
+    ctx->device = device;
+    ctx->n_sm = n_sm;
+    ctx->attn_kernel = 0;
+    ctx->ev_start = ctx->ev_stop = nullptr;
+    reader_status st = sm100_host_init(&ctx->sm100, device);
+    if (st != READER_OK) {
+        delete ctx;
+        return st;
+    }
+    *out = ctx;
+    return READER_OK;
+}
+
+void reader_destroy(reader_ctx *ctx) { delete ctx; }
+
+const char *reader_status_string(reader_status s) {
+    switch (s) {
+        case READER_OK: return "ok";
+        case READER_ERR_INVALID_ARG: return "invalid argument";
+        case READER_ERR_BAD_TREE: return "parent array is not a tree rooted at node 0 with parent[j] < j";
+        case READER_ERR_CAPACITY: return "page table cannot hold the requested positions";
+        case READER_ERR_WORKSPACE: return "workspace too small";
+        case READER_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case READER_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case READER_ERR_CUDA: return "CUDA call failed";
+        case READER_ERR_BAD_PAGE: return "page id outside the pool";
+    }
+    return "unknown status";
+}
+
+reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which) {
+    if (!ctx || which < 0 || which > 2) return READER_ERR_INVALID_ARG;
+    ctx->attn_kernel = which;
+    return READER_OK;
+}
+
+reader_status reader_set_timing_events(reader_ctx *ctx, void *start, void *stop) {
+    if (!ctx || ((start == nullptr) != (stop == nullptr))) return READER_ERR_INVALID_ARG;
+    ctx->ev_start = (cudaEvent_t)start;
+    ctx->ev_stop = (cudaEvent_t)stop;
+    return READER_OK;
+}
+
+size_t reader_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes, int32_t n_q_heads,
+                              int32_t n_kv_heads, int32_t head_dim) {
+    if (!ctx || !shape_ok(max_batch, max_nodes, n_q_heads, n_kv_heads, head_dim)) return 0;
+    return ws_layout(ctx, max_batch, max_nodes, head_dim).total;
+}
+
+reader_status reader_tree_encode(reader_ctx *ctx, const int32_t *parent, int32_t batch, int32_t n_nodes,
+                                 uint64_t *anc_mask_out, int32_t *level_out, int32_t *status_out, void *stream) {
+    if (!ctx || !parent || !anc_mask_out || !status_out || batch < 0 || n_nodes < 1 || n_nodes > kMaxNodes ||
+        !aligned16(anc_mask_out))
+        return READER_ERR_INVALID_ARG;
+    if (reader_status st = check_device(ctx)) return st;
+    launch_tree_encode(parent, batch, n_nodes, anc_mask_out, level_out, status_out, (cudaStream_t)stream);
+    return launch_status();
+}
+
+reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
+                                 const void *v_tree, const reader_kv_cache *cache, const reader_tree *tree,
+                                 float softmax_scale, void *out, float *lse_out, void *workspace,
+                                 size_t workspace_bytes, int32_t *status_out, void *stream) {
+    if (!ctx || !q || !k_tree || !v_tree || !cache || !tree || !out || !workspace || !status_out)
+        return READER_ERR_INVALID_ARG;
+    const int B = tree->batch, T = tree->n_nodes, Hq = n_q_heads, Hkv = cache->n_kv_heads, D = cache->head_dim;
+    if (!cache->k_pool || !cache->v_pool || !cache->page_table || !cache->seq_lens || !tree->parent)
+        return READER_ERR_INVALID_ARG;
+    if (B < 0 || T < 1 || T > kMaxNodes || Hq < 1 || Hkv < 1 || cache->num_pages < 0 ||
+        cache->max_pages_per_seq < 1 || !(softmax_scale == softmax_scale))
+        return READER_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128) || cache->page_size != kPage) return READER_ERR_UNSUPPORTED;
+    if (cache->shared_prefix_len < 0 || cache->shared_prefix_len % kPage != 0) return READER_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k_pool) ||
+        !aligned16(cache->v_pool) || !aligned16(out) || !aligned16(tree->anc_mask) ||
+        (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0)
+        return READER_ERR_INVALID_ARG;
+    const int G = Hq / Hkv;
+    const int n_mtiles = (T * G + kTileM - 1) / kTileM;
+    const int n_tree_tiles = (T + kPage - 1) / kPage;
+    const int64_t tiles_bound = (int64_t)B * Hkv * n_mtiles * ((int64_t)cache->max_pages_per_seq + n_tree_tiles);
+    if (tiles_bound >= (int64_t)1 << 31) return READER_ERR_UNSUPPORTED;
+    const WsLayout w = ws_layout(ctx, B, T, D);
+    if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
+    if (reader_status st = check_device(ctx)) return st;
+    if (B == 0) return READER_OK;
+
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = (cudaStream_t)stream;
+
+    AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.k_tree = static_cast<const __nv_bfloat16 *>(k_tree);
+    p.v_tree = static_cast<const __nv_bfloat16 *>(v_tree);
+    p.k_pool = static_cast<const __nv_bfloat16 *>(cache->k_pool);
+    p.v_pool = static_cast<const __nv_bfloat16 *>(cache->v_pool);
+    p.page_table = cache->page_table;
+    p.seq_lens = cache->seq_lens;
+    p.anc = tree->anc_mask ? tree->anc_mask : reinterpret_cast<const uint64_t *>(ws + w.anc);
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse_out;
+    p.partial_o = reinterpret_cast<float *>(ws + w.partial_o);
+    p.partial_ml = reinterpret_cast<float *>(ws + w.partial_ml);
+    p.status = status_out;
+    p.error_flag = reinterpret_cast<int32_t *>(ws + w.error_flag);
+    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = G;
+    p.max_pages = cache->max_pages_per_seq;
+    p.num_pages = cache->num_pages;
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.sched.seq_tile_start = reinterpret_cast<const int32_t *>(ws + w.seq_tile_start);
+    p.sched.seq_ntiles = reinterpret_cast<const int32_t *>(ws + w.seq_ntiles);
+    p.sched.seq_npages = reinterpret_cast<const int32_t *>(ws + w.seq_npages);
+    p.sched.units_per_seq = Hkv * n_mtiles;
+    p.sched.n_mtiles = n_mtiles;
+
+    const bool tc_ok = sm100_supports(&ctx->sm100, p);
+    if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
+    const bool use_tc = tc_ok && ctx->attn_kernel != 1;
+    p.sched.n_ctas = use_tc ? ctx->n_sm : max_ctas(ctx);
+
+    launch_prepare(*cache, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
+                   tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
+                   reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
+                   reinterpret_cast<int32_t *>(ws + w.seq_npages), status_out, p.error_flag, st);
+    if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
+    if (use_tc) {
+        if (reader_status s = launch_attn_sm100(&ctx->sm100, p, *cache, st)) return s;
+    } else {
+        launch_attn_generic(p, st);
+    }
+    if (ctx->ev_stop) cudaEventRecord(ctx->ev_stop, st);
+    launch_combine(p, st);
+    return launch_status();
+}
+
+reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens,
+                            const float *logits, int32_t vocab, int32_t *target_ids, int32_t max_path,
+                            int32_t *path_out, int32_t *n_acc_out, int32_t *bonus_out, void *workspace,
+                            size_t workspace_bytes, int32_t *status_out, void *stream) {
+    if (!ctx || !tree || !tree->parent || !node_tokens || !target_ids || !path_out || !n_acc_out || !bonus_out ||
+        !status_out)
+        return READER_ERR_INVALID_ARG;
+    const int B = tree->batch, T = tree->n_nodes;
+    if (B < 0 || T < 1 || T > kMaxNodes || max_path < 1) return READER_ERR_INVALID_ARG;
+    if (reader_status st = check_device(ctx)) return st;
+    if (B == 0) return READER_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    int splits = 0;
+    float *pv = nullptr;
+    int32_t *pi = nullptr;
+    if (logits) {
+        if (vocab < 1 || !workspace || !aligned16(logits) || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0)
+            return READER_ERR_INVALID_ARG;
+        // only the argmax regions are used, so any head shape that sized the workspace will do
+        const WsLayout w = ws_layout(ctx, B, T, 64);
+        if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
+        const int64_t rows = (int64_t)B * T;
+        int64_t want = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;
+        int64_t cap = vocab / 2048 > 0 ? vocab / 2048 : 1;
+        splits = (int)(want < 1 ? 1 : want);
+        if (splits > cap) splits = (int)cap;
+        if (splits > kMaxSplits) splits = kMaxSplits;
+        unsigned char *ws = static_cast<unsigned char *>(workspace);
+        pv = reinterpret_cast<float *>(ws + w.amax_val);
+        pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);
+        launch_argmax(logits, rows, vocab, splits, pv, pi, st);
+    }
+    launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, pv, pi, splits, path_out, n_acc_out,
+                  bonus_out, status_out, st);
+    return launch_status();
+}
+
+reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const void *k_tree, const void *v_tree,
+                               int32_t batch, int32_t n_nodes, const int32_t *path, const int32_t *n_acc,
+                               int32_t max_path, int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out,
+                               void *stream) {
+    if (!ctx || !cache || !k_tree || !v_tree || !path || !n_acc || !slots_out || !status_out ||
+        !cache->k_pool || !cache->v_pool || !cache->page_table || !cache->seq_lens)
+        return READER_ERR_INVALID_ARG;
+    if (batch < 0 || n_nodes < 1 || n_nodes > kMaxNodes || max_path < 1 || cache->n_kv_heads < 1 ||
+        cache->max_pages_per_seq < 1 || cache->num_pages < 0 || cache->shared_prefix_len < 0 ||
+        cache->shared_prefix_len % kPage != 0)
+        return READER_ERR_INVALID_ARG;
+    if (cache->page_size != kPage || cache->head_dim % 8 != 0 || cache->head_dim < 8) return READER_ERR_UNSUPPORTED;
+    if (!aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k_pool) || !aligned16(cache->v_pool))
+        return READER_ERR_INVALID_ARG;
+    if (reader_status st = check_device(ctx)) return st;
+    launch_kv_commit(*cache, static_cast<const __nv_bfloat16 *>(k_tree), static_cast<const __nv_bfloat16 *>(v_tree),
+                     batch, n_nodes, path, n_acc, max_path, update_seq_lens, slots_out, status_out,
+                     (cudaStream_t)stream);
+    return launch_status();
+}
+
+}  // extern "C"

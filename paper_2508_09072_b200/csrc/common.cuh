@@ -1,0 +1,125 @@
+// Shared declarations of the verification kernels: parameter blocks, the flattened
+// split-KV work partition, and small device helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "reader_verify.h"
+
+namespace reader {
+
+constexpr int kPage = READER_PAGE_SIZE;   // tokens per KV tile (= cache page)
+constexpr int kTileM = 128;               // query rows per M tile
+constexpr int kMaxNodes = READER_MAX_NODES;
+
+// ---------------------------------------------------------------------------------------------
+// Work partition (split-KV over a flattened tile list).
+//
+// A *unit* is (sequence b, KV head h, M tile mt): kTileM query rows (node j, group member g) with
+// row = j * G + g, attending over ntiles(b) KV tiles: the committed pages of b followed by the
+// tree tiles.  Units are ordered (b, h, mt), tiles within a unit in order, and the resulting flat
+// list of W tiles is cut into n_ctas contiguous ranges of near-equal length.  The part of a
+// range that lies in one unit is a *segment*.  A segment that covers its whole unit writes the
+// final output; any other segment writes an (m, l, O) partial into one of the CTA's two slots:
+// slot 2c when the segment does not start its unit, slot 2c+1 when it does.
+// ---------------------------------------------------------------------------------------------
+struct Sched {
+    const int32_t *seq_tile_start;  // [B+1] first flat tile of sequence b
+    const int32_t *seq_ntiles;      // [B]   tiles per unit of sequence b (0: sequence skipped)
+    const int32_t *seq_npages;      // [B]   committed pages among them
+    int32_t n_ctas;
+    int32_t units_per_seq;          // Hkv * n_mtiles
+    int32_t n_mtiles;
+};
+
+struct Segment {
+    int b, h, mt;
+    int tile_begin, tile_end;  // within the unit
+    int ntiles, npages;
+    bool full;                 // covers the whole unit
+    int slot;                  // partial slot when !full
+};
+
+__device__ __forceinline__ int range_begin(int c, int n_ctas, int W) {
+    return (int)(((int64_t)c * W) / n_ctas);
+}
+
+// Largest b with seq_tile_start[b] <= w (w < W).
+__device__ __forceinline__ int find_seq(const int32_t *start, int B, int w) {
+    int lo = 0, hi = B;  // invariant: start[lo] <= w < start[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (start[mid] <= w) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ Segment segment_at(const Sched &s, int B, int cta, int w, int range_end) {
+    Segment g;
+    g.b = find_seq(s.seq_tile_start, B, w);
+    g.ntiles = s.seq_ntiles[g.b];
+    g.npages = s.seq_npages[g.b];
+    int local = w - s.seq_tile_start[g.b];
+    int unit = local / g.ntiles;
+    g.tile_begin = local - unit * g.ntiles;
+    g.h = unit / s.n_mtiles;
+    g.mt = unit - g.h * s.n_mtiles;
+    int left = range_end - w;
+    g.tile_end = min(g.ntiles, g.tile_begin + left);
+    g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
+    g.slot = 2 * cta + (g.tile_begin == 0 ? 1 : 0);
+    return g;
+}
+
+// CTA whose range contains flat tile w.
+__device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
+    int c = (int)(((int64_t)w * n_ctas) / W);
+    if (c >= n_ctas) c = n_ctas - 1;
+    while (c + 1 < n_ctas && range_begin(c + 1, n_ctas, W) <= w) ++c;
+    while (c > 0 && range_begin(c, n_ctas, W) > w) --c;
+    return c;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention parameters
+// ---------------------------------------------------------------------------------------------
+struct AttnParams {
+    const __nv_bfloat16 *q, *k_tree, *v_tree, *k_pool, *v_pool;
+    const int32_t *page_table;
+    const int32_t *seq_lens;
+    const uint64_t *anc;       // [B][T][2]
+    __nv_bfloat16 *out;
+    float *lse;                // nullable
+    float *partial_o;          // [slots][kTileM][D]
+    float *partial_ml;         // [slots][kTileM][2]  (m in log2 units, l)
+    int32_t *status;           // [B]
+    int32_t *error_flag;       // one word in the workspace: set on a bounded-wait timeout
+    int B, T, Hq, Hkv, D, G;
+    int max_pages, num_pages;
+    float scale_log2;          // softmax_scale * log2(e)
+    Sched sched;
+};
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// Host-side launchers (one per .cu file)
+void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int32_t *level,
+                        int32_t *status, cudaStream_t st);
+void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
+                    int units_per_seq, uint64_t *anc_out /*nullable*/, int32_t *seq_tile_start,
+                    int32_t *seq_ntiles, int32_t *seq_npages, int32_t *status, int32_t *error_flag,
+                    cudaStream_t st);
+void launch_attn_generic(const AttnParams &p, cudaStream_t st);
+void launch_combine(const AttnParams &p, cudaStream_t st);
+void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits, float *part_val,
+                   int32_t *part_idx, cudaStream_t st);
+void launch_accept(const int32_t *parent, const int32_t *tok, int32_t *target, int B, int T,
+                   int max_path, const float *part_val, const int32_t *part_idx, int splits,
+                   int32_t *path, int32_t *n_acc, int32_t *bonus, int32_t *status, cudaStream_t st);
+void launch_kv_commit(const reader_kv_cache &c, const __nv_bfloat16 *k_tree, const __nv_bfloat16 *v_tree,
+                      int B, int T, const int32_t *path, const int32_t *n_acc, int max_path,
+                      int update_seq_lens, int32_t *slots, int32_t *status, cudaStream_t st);
+
+}  // namespace reader

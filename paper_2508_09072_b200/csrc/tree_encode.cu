@@ -1,0 +1,113 @@
+// Tree-mask encoder (Sec. 3.2: M_ij = 1 iff node i is an ancestor of node j, made reflexive) and
+// the per-call preparation kernel that validates every sequence and lays out the split-KV work.
+#include "common.cuh"
+#include "tree.cuh"
+
+namespace reader {
+
+__global__ void __launch_bounds__(128) tree_encode_kernel(const int32_t *__restrict__ parent, int B, int T,
+                                                          uint64_t *__restrict__ anc, int32_t *__restrict__ level,
+                                                          int32_t *__restrict__ status) {
+    __shared__ int32_t par[4][kMaxNodes];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 4 + warp;
+    if (b >= B) return;
+    for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];
+    __syncwarp();
+    const bool ok = warp_tree_valid(par[warp], T, lane);
+    for (int j = lane; j < T; j += 32) {
+        uint64_t lo = 0, hi = 0;
+        int lv = 0;
+        if (ok) node_ancestors(par[warp], T, j, lo, hi, lv);
+        anc[((size_t)b * T + j) * 2 + 0] = lo;
+        anc[((size_t)b * T + j) * 2 + 1] = hi;
+        if (level) level[(size_t)b * T + j] = lv;
+    }
+    if (lane == 0) status[b] = ok ? READER_OK : READER_ERR_BAD_TREE;
+}
+
+void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int32_t *level,
+                        int32_t *status, cudaStream_t st) {
+    if (B <= 0) return;
+    tree_encode_kernel<<<(B + 3) / 4, 128, 0, st>>>(parent, B, T, anc, level, status);
+}
+
+// One CTA.  Each warp takes sequences b = warp, warp + 32, ...: checks the tree (encoding the
+// masks when asked), the committed length against the page table's capacity and every page id
+// in use; then warp 0 turns the per-sequence tile counts into the flat prefix the attention
+// kernels cut into CTA ranges.
+__global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict__ page_table,
+                                                       const int32_t *__restrict__ seq_lens, int max_pages,
+                                                       int num_pages, const int32_t *__restrict__ parent, int B,
+                                                       int T, int n_tree_tiles, int units_per_seq,
+                                                       uint64_t *__restrict__ anc_out,
+                                                       int32_t *__restrict__ seq_tile_start,
+                                                       int32_t *__restrict__ seq_ntiles,
+                                                       int32_t *__restrict__ seq_npages,
+                                                       int32_t *__restrict__ status,
+                                                       int32_t *__restrict__ error_flag) {
+    __shared__ int32_t par[32][kMaxNodes];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) *error_flag = 0;
+    for (int b = warp; b < B; b += 32) {
+        for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];
+        __syncwarp();
+        int st = warp_tree_valid(par[warp], T, lane) ? READER_OK : READER_ERR_BAD_TREE;
+        if (anc_out) {
+            for (int j = lane; j < T; j += 32) {
+                uint64_t lo = 0, hi = 0;
+                int lv = 0;
+                if (st == READER_OK) node_ancestors(par[warp], T, j, lo, hi, lv);
+                anc_out[((size_t)b * T + j) * 2 + 0] = lo;
+                anc_out[((size_t)b * T + j) * 2 + 1] = hi;
+            }
+        }
+        const int L = seq_lens[b];
+        int npages = 0;
+        if (st == READER_OK) {
+            if (L < 0 || (int64_t)L > (int64_t)max_pages * kPage) {
+                st = READER_ERR_CAPACITY;
+            } else {
+                npages = (L + kPage - 1) / kPage;
+                bool ok = true;
+                for (int p = lane; p < npages; p += 32) {
+                    int pg = page_table[(size_t)b * max_pages + p];
+                    ok = ok && pg >= 0 && pg < num_pages;
+                }
+                if (!__all_sync(0xffffffffu, ok)) st = READER_ERR_BAD_PAGE;
+            }
+        }
+        if (lane == 0) {
+            status[b] = st;
+            seq_ntiles[b] = st == READER_OK ? npages + n_tree_tiles : 0;
+            seq_npages[b] = st == READER_OK ? npages : 0;
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        if (lane == 0) seq_tile_start[0] = 0;
+        for (int base = 0; base < B; base += 32) {
+            int b = base + lane;
+            int v = b < B ? seq_ntiles[b] * units_per_seq : 0;
+            int incl = v;
+            for (int d = 1; d < 32; d <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += t;
+            }
+            if (b < B) seq_tile_start[b + 1] = carry + incl;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+}
+
+void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
+                    int units_per_seq, uint64_t *anc_out, int32_t *seq_tile_start, int32_t *seq_ntiles,
+                    int32_t *seq_npages, int32_t *status, int32_t *error_flag, cudaStream_t st) {
+    prepare_kernel<<<1, 1024, 0, st>>>(c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages, parent, B, T,
+                                       n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles,
+                                       seq_npages, status, error_flag);
+}
+
+}  // namespace reader

@@ -3,7 +3,7 @@
 This module only *draws inputs*: tree shapes, bf16 tensors, page tables, token
 ids and logits.  It holds none of the method's arithmetic (no attention, no
 acceptance rule, no commit) and imports neither the CUDA binding nor the CPU
-oracle, so both sides can be fed the very same arrays.
+checker used by the tests, so both sides can be fed the very same arrays.
 
 The five named workloads C1..C5 are synthetic stand-ins for the public suites
 and trained 7-8B models the paper evaluates on (Sec. 5): none of those is

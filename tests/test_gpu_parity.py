@@ -1,0 +1,375 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs.
+
+Integer results (masks, levels, argmax, paths, lengths, bonus tokens, slots, the whole KV pool,
+seq_lens, status words) must match bit for bit.  Attention outputs (bf16 inputs, fp32
+accumulation, bf16 output) must be within max abs error 2e-2 and mean abs error 2e-3 of the fp64
+oracle; log-sum-exp within 2e-3.
+"""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2508_09072_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS, LSE_ABS = 2e-2, 2e-3, 2e-3
+
+
+@pytest.fixture(scope="module")
+def rd():
+    from paper_2508_09072_b200 import binding
+    r = binding.Reader(0)
+    yield r
+    r.close()
+
+
+def gpu_attn(rd, w, kernel=0, pre_encode=False, want_lse=True):
+    from paper_2508_09072_b200 import binding
+    d = binding.to_device(w, with_logits=False)
+    rd.set_attn_kernel(kernel)
+    anc = None
+    if pre_encode:
+        anc, _, _ = rd.tree_encode(d.parent)
+    lse = torch.full((w.batch, w.n_nodes, w.n_q_heads), 7.0, dtype=torch.float32, device="cuda") if want_lse else None
+    out = torch.full((w.batch, w.n_nodes, w.n_q_heads, w.head_dim), 3.0, dtype=torch.bfloat16, device="cuda")
+    out, status = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out, lse=lse)
+    torch.cuda.synchronize()
+    rd.set_attn_kernel(0)
+    o = W.bf16_bits_to_f32(binding.bf16_bits(out)).astype(np.float64)
+    return o, status.cpu().numpy(), (lse.cpu().numpy().astype(np.float64) if want_lse else None)
+
+
+def check_attn(w, got, status, lse, ref=None):
+    ref = ref or oracle.verify_attn(w.q, w.k_tree, w.v_tree, w.k_pool, w.v_pool, w.page_table, w.seq_lens,
+                                    w.parent, w.scale, want_lse=True)
+    np.testing.assert_array_equal(status, ref["status"])
+    err = np.abs(got - ref["out"])
+    assert np.isfinite(got).all()
+    assert err.max() <= MAX_ABS, f"max abs err {err.max()}"
+    assert err.mean() <= MEAN_ABS, f"mean abs err {err.mean()}"
+    if lse is not None:
+        assert np.abs(lse - ref["lse"]).max() <= LSE_ABS
+    return err.max(), err.mean()
+
+
+def sub_workload(w, b, hk):
+    """Sequence b, KV head hk of a workload as a batch-1, one-KV-head problem (for sampled checks)."""
+    G = w.n_q_heads // w.n_kv_heads
+    s = copy.copy(w)
+    s.batch, s.n_q_heads, s.n_kv_heads = 1, G, 1
+    s.q = np.ascontiguousarray(w.q[b:b + 1, :, hk * G:(hk + 1) * G])
+    s.k_tree = np.ascontiguousarray(w.k_tree[b:b + 1, :, hk:hk + 1])
+    s.v_tree = np.ascontiguousarray(w.v_tree[b:b + 1, :, hk:hk + 1])
+    used = w.page_table[b][w.page_table[b] >= 0]
+    remap = np.full(w.num_pages, -1, np.int32)
+    remap[used] = np.arange(len(used), dtype=np.int32)
+    s.k_pool = np.ascontiguousarray(w.k_pool[used, hk:hk + 1])
+    s.v_pool = np.ascontiguousarray(w.v_pool[used, hk:hk + 1])
+    s.page_table = np.where(w.page_table[b:b + 1] >= 0, remap[np.maximum(w.page_table[b:b + 1], 0)], -1).astype(np.int32)
+    s.seq_lens = w.seq_lens[b:b + 1].copy()
+    s.parent = w.parent[b:b + 1].copy()
+    return s
+
+
+# ------------------------------------------------------------------------------------ tree encode
+@pytest.mark.parametrize("T", [1, 2, 31, 64, 65, 128])
+def test_tree_encode_matches_oracle(rd, T):
+    rng = np.random.default_rng(T)
+    trees = [W.chain_tree(T), W.star_tree(T)] + [W.capped_recursive_tree(rng, T, 12, 4) for _ in range(7)]
+    parent = np.stack(trees).astype(np.int32)
+    bad = parent.copy()
+    if T > 2:
+        bad[1, T - 1] = T - 1          # self parent
+        bad[2, 0] = 0                  # root with a parent
+    anc, level, status = rd.tree_encode(torch.from_numpy(bad).cuda())
+    torch.cuda.synchronize()
+    anc = anc.cpu().numpy().view(np.uint64)
+    for b in range(len(trees)):
+        if not oracle.tree_is_valid(bad[b]):
+            assert status[b].item() == oracle.BAD_TREE and not anc[b].any()
+            continue
+        assert status[b].item() == 0
+        M = oracle.ancestor_matrix(bad[b])
+        bits = np.zeros((T, T), np.uint8)
+        for j in range(T):
+            for i in range(T):
+                bits[i, j] = (int(anc[b, j, i // 64]) >> (i % 64)) & 1
+        np.testing.assert_array_equal(bits, M)
+        np.testing.assert_array_equal(level[b].cpu().numpy(), oracle.levels(bad[b]))
+
+
+# ------------------------------------------------------------------------------------ attention
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("name", W.WORKLOADS)
+def test_attn_named_workloads_small(rd, name, kernel):
+    w = W.make(name, with_logits=False, reduced=(name != "c1"))
+    got, status, lse = gpu_attn(rd, w, kernel=kernel)
+    check_attn(w, got, status, lse)
+
+
+SHAPES = [
+    # T, Hq, Hkv, D, lens
+    (1, 8, 8, 64, (0, 1, 63, 64, 65)),
+    (5, 4, 4, 128, (0, 200)),
+    (33, 8, 2, 128, (130, 7, 450)),
+    (64, 16, 2, 64, (129,)),
+    (128, 8, 2, 128, (70, 300)),
+    (100, 6, 2, 64, (90,)),         # group of 3: CUDA-core kernel only
+    (17, 32, 8, 128, (1000, 513, 64)),
+    (128, 32, 8, 128, (777,)),
+]
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("case", range(len(SHAPES)))
+def test_attn_shapes_and_ragged_lengths(rd, case, kernel):
+    T, Hq, Hkv, D, lens = SHAPES[case]
+    w = W.build_workload("s", 900 + case, list(lens), T, Hq, Hkv, D,
+                         lambda r: W.capped_recursive_tree(r, T, 12, 4), max_path=12, vocab=16,
+                         shuffle_pages=True, with_logits=False, spare_pages=3)
+    got, status, lse = gpu_attn(rd, w, kernel=kernel, pre_encode=(case % 2 == 0))
+    check_attn(w, got, status, lse)
+
+
+def test_attn_many_short_sequences_and_widened_trees(rd):
+    rng = np.random.default_rng(77)
+    lens = rng.integers(0, 200, size=40)
+    w = W.build_workload("s", 78, lens, 24, 8, 2, 128, lambda r: W.widened_tree(r, 24, 10, 4, 3), max_path=11,
+                         vocab=16, shuffle_pages=True, with_logits=False)
+    got, status, lse = gpu_attn(rd, w)
+    check_attn(w, got, status, lse)
+
+
+def test_attn_status_words_and_poisoned_tail(rd):
+    w = W.build_workload("s", 81, [100, 70, 150, 64], 12, 8, 2, 128, lambda r: W.capped_recursive_tree(r, 12, 5, 3),
+                         max_path=5, vocab=16, shuffle_pages=True, with_logits=False)
+    w.parent[1, 5] = 7                                   # forward parent
+    w.page_table[2, 1] = w.num_pages + 3                 # page id outside the pool
+    pg = w.page_table[0, 1]
+    w.k_pool[pg, :, 36:, :] = 0x7FC0                     # NaN / inf beyond seq_len 100 on its last page
+    w.v_pool[pg, :, 36:, :] = 0x7F80
+    for kernel in (0, 1):
+        got, status, lse = gpu_attn(rd, w, kernel=kernel)
+        assert status.tolist() == [0, oracle.BAD_TREE, oracle.BAD_PAGE, 0]
+        assert not got[1].any() and not got[2].any() and not lse[1].any() and not lse[2].any()
+        check_attn(w, got, status, lse)
+    w.seq_lens[3] = w.max_pages * 64 + 1
+    got, status, _ = gpu_attn(rd, w)
+    assert status[3] == oracle.CAPACITY and not got[3].any()
+
+
+def test_attn_shared_prefix_equals_duplicated_prefix(rd):
+    w = W.make("c5", with_logits=False, reduced=True)
+    a, _, _ = gpu_attn(rd, w)
+    b, _, _ = gpu_attn(rd, W.duplicate_shared_prefix(w))
+    err = np.abs(a - b)
+    assert err.max() <= 2 ** -6          # the split points differ, so only rounding-level differences
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+def test_attn_full_size_sampled_against_oracle(rd, name):
+    """BASELINE sizes in the launch configuration the benchmark times; the oracle recomputes
+    sampled (sequence, KV head) slices one by one."""
+    w = W.make(name, with_logits=False)
+    got, status, lse = gpu_attn(rd, w)
+    assert not status.any() and np.isfinite(got).all()
+    rng = np.random.default_rng(5)
+    G = w.n_q_heads // w.n_kv_heads
+    n_samples = 2 if name == "c4" else 4
+    for _ in range(n_samples):
+        b, hk = int(rng.integers(w.batch)), int(rng.integers(w.n_kv_heads))
+        s = sub_workload(w, b, hk)
+        check_attn(s, got[b:b + 1, :, hk * G:(hk + 1) * G], status[b:b + 1], lse[b:b + 1, :, hk * G:(hk + 1) * G])
+
+
+# ------------------------------------------------------------------------------------ acceptance
+def gpu_accept(rd, w, use_logits=True, target=None, max_path=None):
+    d_parent = torch.from_numpy(w.parent).cuda()
+    d_tok = torch.from_numpy(w.node_tokens).cuda()
+    kw = {}
+    if use_logits:
+        kw["logits"] = torch.from_numpy(w.logits).cuda()
+    else:
+        kw["target_ids"] = torch.from_numpy(target).cuda()
+    r = rd.accept(d_parent, d_tok, max_path or w.max_path, **kw)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in r.items()}
+
+
+def check_accept(w, got, max_path=None):
+    tgt = oracle.argmax(w.logits)
+    np.testing.assert_array_equal(got["target_ids"], tgt)
+    ref = oracle.accept(w.parent, w.node_tokens, tgt, max_path or w.max_path)
+    for k in ("path", "n_acc", "bonus", "status"):
+        np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+    return ref
+
+
+@pytest.mark.parametrize("name", W.WORKLOADS)
+def test_accept_named_workloads_small(rd, name):
+    w = W.make(name, reduced=(name != "c1"))
+    ref = check_accept(w, gpu_accept(rd, w))
+    assert np.all(ref["n_acc"] >= w.planted_len)
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_accept_full_size(rd, name):
+    w = W.make(name)
+    check_accept(w, gpu_accept(rd, w))
+
+
+def test_argmax_ties_nan_and_odd_vocab(rd):
+    rng = np.random.default_rng(3)
+    for vocab in (1, 7, 1000, 4099, 8192):
+        T = 9
+        w = W.build_workload("s", vocab, [10, 20, 30], T, 2, 1, 64, lambda r: W.capped_recursive_tree(r, T, 5, 3),
+                             max_path=5, vocab=vocab, shuffle_pages=False, zipf_tokens=False)
+        lg = rng.integers(0, 4, size=w.logits.shape).astype(np.float32)      # heavy ties
+        if vocab > 1:
+            lg[0, 0, 0] = np.nan
+            lg[0, 1, :] = np.nan
+            lg[0, 2, :] = -np.inf
+            lg[1, 3, vocab // 2] = np.nan
+            lg[1, 4, vocab - 1] = np.inf
+        w.logits = lg
+        check_accept(w, gpu_accept(rd, w))
+
+
+def test_accept_exhaustive_small_trees_with_given_targets(rd):
+    import itertools
+    T, vocab = 5, 3
+    combos = np.array(list(itertools.product(range(vocab), repeat=T)), dtype=np.int32)
+    n = len(combos)
+    tok = np.repeat(combos, n, axis=0)
+    tgt = np.tile(combos, (n, 1))
+    for tail in itertools.product(*[range(j) for j in range(1, T)]):
+        parent = np.broadcast_to(np.array((-1,) + tail, np.int32), tok.shape).copy()
+        w = type("X", (), {})()
+        w.parent, w.node_tokens, w.max_path = parent, tok, T
+        for mp in (T, 2):
+            got = gpu_accept(rd, w, use_logits=False, target=tgt, max_path=mp)
+            ref = oracle.accept(parent, tok, tgt, mp)
+            for k in ("path", "n_acc", "bonus", "status"):
+                np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+
+
+def test_accept_big_trees_duplicates_and_bad_tree(rd):
+    rng = np.random.default_rng(9)
+    B, T = 200, 128
+    parent = np.stack([W.widened_tree(rng, T, 40, 8, 4) if b % 2 else W.capped_recursive_tree(rng, T, 12, 4)
+                       for b in range(B)])
+    tok = rng.integers(0, 3, size=(B, T)).astype(np.int32)      # tiny vocabulary: many equal siblings, long matches
+    tgt = rng.integers(0, 3, size=(B, T)).astype(np.int32)
+    parent[7, 9] = 9
+    parent[8, 0] = 3
+    w = type("X", (), {})()
+    w.parent, w.node_tokens = parent, tok
+    for mp in (128, 12, 1):
+        got = gpu_accept(rd, w, use_logits=False, target=tgt, max_path=mp)
+        ref = oracle.accept(parent, tok, tgt, mp)
+        for k in ("path", "n_acc", "bonus", "status"):
+            np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+    assert ref["status"][7] == oracle.BAD_TREE and ref["status"][8] == oracle.BAD_TREE
+
+
+# ------------------------------------------------------------------------------------ commit
+def gpu_commit(rd, w, path, n_acc, update=True):
+    from paper_2508_09072_b200 import binding
+    d = binding.to_device(w, with_logits=False)
+    slots, status = rd.kv_commit(d.cache, d.k_tree, d.v_tree, torch.from_numpy(path).cuda(),
+                                 torch.from_numpy(n_acc).cuda(), update_seq_lens=update)
+    torch.cuda.synchronize()
+    return {"k_pool": binding.bf16_bits(d.cache.k_pool), "v_pool": binding.bf16_bits(d.cache.v_pool),
+            "seq_lens": d.cache.seq_lens.cpu().numpy(), "slots": slots.cpu().numpy(), "status": status.cpu().numpy()}
+
+
+def check_commit(w, path, n_acc, update=True):
+    ref = oracle.kv_commit(w.k_pool, w.v_pool, w.page_table, w.seq_lens, w.shared_prefix_len, w.k_tree, w.v_tree,
+                           path, n_acc, update_seq_lens=update)
+    return ref
+
+
+@pytest.mark.parametrize("name", W.WORKLOADS)
+def test_commit_named_workloads_small(rd, name):
+    w = W.make(name, reduced=(name != "c1"))
+    a = oracle.accept(w.parent, w.node_tokens, oracle.argmax(w.logits), w.max_path)
+    for update in (True, False):
+        got = gpu_commit(rd, w, a["path"], a["n_acc"], update)
+        ref = check_commit(w, a["path"], a["n_acc"], update)
+        for k in ("k_pool", "v_pool", "seq_lens", "slots", "status"):
+            np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+
+
+def test_commit_page_crossing_capacity_and_prefix_guard(rd):
+    T = 20
+    w = W.build_workload("s", 31, [60, 127, 200, 128 + 5, 64], T, 8, 4, 64,
+                         lambda r: W.chain_tree(T), max_path=16, vocab=16, shuffle_pages=True, with_logits=False,
+                         spare_pages=2)
+    path = np.tile(np.arange(16, dtype=np.int32), (5, 1))
+    n_acc = np.array([16, 9, 0, 3, 16], np.int32)
+    w.page_table[1, 2:] = -1                     # sequence 1 has no page for positions >= 128
+    w.shared_prefix_len = 0
+    got = gpu_commit(rd, w, path, n_acc)
+    ref = check_commit(w, path, n_acc)
+    assert ref["status"].tolist() == [0, oracle.CAPACITY, 0, 0, 0]
+    for k in ("k_pool", "v_pool", "seq_lens", "slots", "status"):
+        np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+    # prefix guard and a node id outside the tree
+    w2 = W.build_workload("s", 32, [128 + 3, 128 + 70], T, 8, 4, 64, lambda r: W.chain_tree(T), max_path=16,
+                          vocab=16, shuffle_pages=True, with_logits=False, shared_prefix_len=128)
+    w2.seq_lens[0] = 100
+    path2 = path[:2].copy()
+    path2[1, 2] = T
+    n2 = np.array([4, 5], np.int32)
+    got = gpu_commit(rd, w2, path2, n2)
+    ref = check_commit(w2, path2, n2)
+    assert ref["status"].tolist() == [oracle.CAPACITY, oracle.CAPACITY]
+    for k in ("k_pool", "v_pool", "seq_lens", "slots", "status"):
+        np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+
+
+# ------------------------------------------------------------------------------------ whole step
+def test_whole_step_then_next_step_sees_committed_rows(rd):
+    """encode -> attention -> accept -> commit on the device, then a second attention call must
+    see the rows just committed (the oracle runs the same two steps on its own copy)."""
+    from paper_2508_09072_b200 import binding
+    w = W.make("c3", reduced=True)
+    d = binding.to_device(w)
+    out1, st1 = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale)
+    acc = rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits)
+    rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc["path"], acc["n_acc"])
+    out2, st2 = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale)
+    torch.cuda.synchronize()
+
+    a = oracle.accept(w.parent, w.node_tokens, oracle.argmax(w.logits), w.max_path)
+    c = oracle.kv_commit(w.k_pool, w.v_pool, w.page_table, w.seq_lens, 0, w.k_tree, w.v_tree, a["path"], a["n_acc"])
+    np.testing.assert_array_equal(d.cache.seq_lens.cpu().numpy(), c["seq_lens"])
+    w2 = copy.copy(w)
+    w2.k_pool, w2.v_pool, w2.seq_lens = c["k_pool"], c["v_pool"], c["seq_lens"]
+    got2 = W.bf16_bits_to_f32(binding.bf16_bits(out2)).astype(np.float64)
+    check_attn(w2, got2, st2.cpu().numpy(), None)
+    got1 = W.bf16_bits_to_f32(binding.bf16_bits(out1)).astype(np.float64)
+    assert np.abs(got1 - got2).max() > 1e-3      # the second step really attended to more keys
+
+
+def test_host_side_argument_errors(rd):
+    from paper_2508_09072_b200 import binding
+    w = W.make("c1", with_logits=False)
+    d = binding.to_device(w, with_logits=False)
+    with pytest.raises(binding.ReaderError) as e:
+        rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale,
+                       workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.ReaderError) as e:
+        rd.verify_attn(d.q[..., :32].contiguous(), d.k_tree[..., :32].contiguous(), d.v_tree[..., :32].contiguous(),
+                       binding.KvCache(d.cache.k_pool[..., :32].contiguous(), d.cache.v_pool[..., :32].contiguous(),
+                                       d.cache.page_table, d.cache.seq_lens), d.parent, w.scale)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.ReaderError) as e:
+        rd.accept(d.parent, d.node_tokens, 0, target_ids=d.node_tokens)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    assert rd.workspace_bytes(4, 129, 8, 8, 64) == 0 and rd.workspace_bytes(4, 16, 8, 3, 64) == 0
