@@ -37,12 +37,14 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
     for (int r = warp; r < rows; r += 4) {
         float mstar = -INFINITY;
         for (int c = c_first; c <= c_last; ++c) {
+            if (range_begin(c + 1, p.sched.n_ctas, W) == range_begin(c, p.sched.n_ctas, W)) continue;  // empty range: wrote nothing
             const int slot = c == c_first ? 2 * c + 1 : 2 * c;
             mstar = fmaxf(mstar, p.partial_ml[((size_t)slot * kTileM + r) * 2]);
         }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float lstar = 0.f;
         for (int c = c_first; c <= c_last; ++c) {
+            if (range_begin(c + 1, p.sched.n_ctas, W) == range_begin(c, p.sched.n_ctas, W)) continue;
             const int slot = c == c_first ? 2 * c + 1 : 2 * c;
             const float2 ml = *reinterpret_cast<const float2 *>(p.partial_ml + ((size_t)slot * kTileM + r) * 2);
             const float wgt = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mstar);

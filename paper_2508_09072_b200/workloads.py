@@ -228,9 +228,11 @@ def plant_accepted_path(rng, parent: np.ndarray, tokens: np.ndarray, logits: np.
     if child_tok and int(np.argmax(logits[e])) in child_tok:
         V = logits.shape[1]
         t = int(rng.integers(V))
-        while t in child_tok:
+        for _ in range(V):              # a vocabulary made of child tokens only has no such token
+            if t not in child_tok:
+                logits[e, t] = logits[e].max() + 1.0
+                break
             t = (t + 1) % V
-        logits[e, t] = logits[e].max() + 1.0
     return want
 
 

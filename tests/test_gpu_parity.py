@@ -36,7 +36,11 @@ def gpu_attn(rd, w, kernel=0, pre_encode=False, want_lse=True):
         anc, _, _ = rd.tree_encode(d.parent)
     lse = torch.full((w.batch, w.n_nodes, w.n_q_heads), 7.0, dtype=torch.float32, device="cuda") if want_lse else None
     out = torch.full((w.batch, w.n_nodes, w.n_q_heads, w.head_dim), 3.0, dtype=torch.bfloat16, device="cuda")
-    out, status = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out, lse=lse)
+    # scratch that a kernel reads without having written it must show: fill it with NaN patterns
+    ws = rd.workspace(max(w.batch, 1), w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    ws.fill_(0xFF)
+    out, status = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out, lse=lse,
+                                 workspace=ws)
     torch.cuda.synchronize()
     rd.set_attn_kernel(0)
     o = W.bf16_bits_to_f32(binding.bf16_bits(out)).astype(np.float64)
@@ -367,7 +371,8 @@ def test_host_side_argument_errors(rd):
     with pytest.raises(binding.ReaderError) as e:
         rd.verify_attn(d.q[..., :32].contiguous(), d.k_tree[..., :32].contiguous(), d.v_tree[..., :32].contiguous(),
                        binding.KvCache(d.cache.k_pool[..., :32].contiguous(), d.cache.v_pool[..., :32].contiguous(),
-                                       d.cache.page_table, d.cache.seq_lens), d.parent, w.scale)
+                                       d.cache.page_table, d.cache.seq_lens), d.parent, w.scale,
+                       workspace=rd.workspace(1, w.n_nodes, w.n_q_heads, w.n_kv_heads, 64))
     assert e.value.code == binding.ERR_UNSUPPORTED
     with pytest.raises(binding.ReaderError) as e:
         rd.accept(d.parent, d.node_tokens, 0, target_ids=d.node_tokens)
