@@ -88,7 +88,11 @@ reader_status reader_create(reader_ctx **out, int device) {
     return READER_OK;
 }
 
-void reader_destroy(reader_ctx *ctx) { delete ctx; }
+void reader_destroy(reader_ctx *ctx) {
+    if (!ctx) return;
+    sm100_host_destroy(&ctx->sm100);
+    delete ctx;
+}
 
 const char *reader_status_string(reader_status s) {
     switch (s) {
@@ -190,7 +194,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.sched.units_per_seq = Hkv * n_mtiles;
     p.sched.n_mtiles = n_mtiles;
 
-    const bool tc_ok = sm100_supports(&ctx->sm100, p);
+    const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
     if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
     const bool use_tc = tc_ok && ctx->attn_kernel != 1;
     p.sched.n_ctas = use_tc ? ctx->n_sm : max_ctas(ctx);

@@ -1,7 +1,8 @@
 // Split-KV combine: merges the (m, l, O) partials of every unit that was cut across CTA ranges,
 //   m* = max_s m_s,  l* = sum_s l_s 2^(m_s - m*),  O = sum_s O_s 2^(m_s - m*) / l*,
 // rounds to bf16 and writes lse = ln 2 * (m* + log2 l*).  Units written directly by the attention
-// kernel are left alone; rows of sequences with a non-zero status are zeroed.
+// kernel are left alone; rows of sequences with a non-zero status are zeroed, and so is every row when the
+// attention kernel raised the error flag (each status word then carries that code).
 #include "common.cuh"
 
 namespace reader {
@@ -18,7 +19,9 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
     const int nt = p.sched.seq_ntiles[b];
     const int rows = min(kTileM, p.T * p.G - mt * kTileM);
 
-    if (nt == 0) {
+    const int err = *p.error_flag;   // a bounded wait gave up somewhere: no row of this call can be trusted
+    if (err != 0 && unit == 0 && threadIdx.x == 0) p.status[b] = err;
+    if (nt == 0 || err != 0) {
         for (int r = warp; r < rows; r += 4) {
             const int grow = mt * kTileM + r;
             const int j = grow / p.G, hq = h * p.G + grow % p.G;

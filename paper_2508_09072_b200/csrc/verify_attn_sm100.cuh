@@ -4,15 +4,19 @@
 
 namespace reader {
 
+struct Sm100Maps;   // cached TMA descriptors of the pool last seen
+
 struct Sm100Host {
     void *encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
     int smem_optin;       // opt-in shared memory per block on the device
-    bool ready;
+    bool ready;           // the kernel can run on this device
+    bool attr_set;        // dynamic shared memory limit raised (done on first launch, device current)
+    Sm100Maps *maps;
 };
 
 reader_status sm100_host_init(Sm100Host *h, int device);
-bool sm100_supports(const Sm100Host *h, const AttnParams &p);
-reader_status launch_attn_sm100(const Sm100Host *h, const AttnParams &p, const reader_kv_cache &cache,
-                                cudaStream_t st);
+void sm100_host_destroy(Sm100Host *h);
+bool sm100_supports(const Sm100Host *h, const AttnParams &p, float softmax_scale);
+reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_kv_cache &cache, cudaStream_t st);
 
 }  // namespace reader
