@@ -197,7 +197,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
     if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
     const bool use_tc = tc_ok && ctx->attn_kernel != 1;
-    p.sched.n_ctas = use_tc ? ctx->n_sm : max_ctas(ctx);
+    p.sched.n_ctas = max_ctas(ctx);   // two resident CTAs per SM for both kernels
 
     launch_prepare(*cache, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
                    tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),

@@ -15,15 +15,16 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
     const int h = unit / p.sched.n_mtiles;
     const int mt = unit - h * p.sched.n_mtiles;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.y * 4 + warp;   // one warp per query row: the merge is latency-bound, so spread it wide
     const int D = p.D;
     const int nt = p.sched.seq_ntiles[b];
     const int rows = min(kTileM, p.T * p.G - mt * kTileM);
 
     const int err = *p.error_flag;   // a bounded wait gave up somewhere: no row of this call can be trusted
-    if (err != 0 && unit == 0 && threadIdx.x == 0) p.status[b] = err;
+    if (err != 0 && unit == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.status[b] = err;
     if (nt == 0 || err != 0) {
-        for (int r = warp; r < rows; r += 4) {
-            const int grow = mt * kTileM + r;
+        if (row < rows) {
+            const int grow = mt * kTileM + row;
             const int j = grow / p.G, hq = h * p.G + grow % p.G;
             __nv_bfloat16 *dst = p.out + (((size_t)b * p.T + j) * p.Hq + hq) * D;
             if (lane * 4 < D) *reinterpret_cast<uint2 *>(dst + lane * 4) = make_uint2(0, 0);
@@ -35,9 +36,10 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
     const int u0 = p.sched.seq_tile_start[b] + unit * nt;
     const int c_first = cta_of_tile(u0, p.sched.n_ctas, W);
     const int c_last = cta_of_tile(u0 + nt - 1, p.sched.n_ctas, W);
-    if (c_first == c_last) return;
+    if (c_first == c_last || row >= rows) return;
 
-    for (int r = warp; r < rows; r += 4) {
+    {
+        const int r = row;
         float mstar = -INFINITY;
         for (int c = c_first; c <= c_last; ++c) {
             if (range_begin(c + 1, p.sched.n_ctas, W) == range_begin(c, p.sched.n_ctas, W)) continue;  // empty range: wrote nothing
@@ -79,7 +81,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
 
 void launch_combine(const AttnParams &p, cudaStream_t st) {
     const int units = p.B * p.sched.units_per_seq;
-    if (units > 0) combine_kernel<<<units, 128, 0, st>>>(p);
+    if (units > 0) combine_kernel<<<dim3(units, kTileM / 4), 128, 0, st>>>(p);
 }
 
 }  // namespace reader

@@ -1,6 +1,6 @@
 // Tree-masked verify attention (Sec. 3.2) on the sm_100a tensor cores.
 //
-// One persistent CTA per SM walks its range of the flattened split-KV tile list.  For every unit
+// Two persistent CTAs per SM each walk their range of the flattened split-KV tile list.  For every unit
 // (sequence, KV head, 128 query rows) it computes S = Q K^T and O += P V with tcgen05.mma, one KV
 // tile of 64 keys (one cache page, or 64 tree nodes) at a time:
 //
@@ -32,7 +32,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kStages = 4;
+constexpr int kStages = 2;          // per CTA; two CTAs share an SM, so four tiles are in flight per SM
 constexpr int kThreads = 192;
 constexpr int kProducerWarp = 4;
 constexpr int kMmaWarp = 5;
@@ -54,7 +54,7 @@ struct Cfg {
     static constexpr int kOffP = kQBytes;
     static constexpr int kOffStages = kOffP + kPBytes;
     static constexpr int kOffBars = kOffStages + kStages * kStageBytes;
-    static constexpr int kSmemBytes = kOffBars + 256 + 1024;   // + barriers + alignment slack
+    static constexpr int kSmemBytes = kOffBars + 256;   // + barriers; two CTAs of head_dim 128 fit one SM
 };
 
 struct Bars {
@@ -82,13 +82,15 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int
 }
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     using C = Cfg<D>;
-    extern __shared__ unsigned char smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    unsigned char *smem = smem_raw + (base - raw);
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t base = smem_u32(smem);
+    if (base & 1023u) {   // the swizzled tiles need 1024-byte alignment; never seen, but checked
+        if (threadIdx.x == 0) atomicExch(p.error_flag, (int32_t)READER_ERR_CUDA);
+        return;
+    }
     Bars *bars = reinterpret_cast<Bars *>(smem + C::kOffBars);
     volatile int32_t *abort_s = &bars->abort;
 
@@ -318,9 +320,13 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                         if (!((hi >> i) & 1u)) s1[i] = 0xff800000u;
                     }
                 }
-                float mx = -INFINITY;
+                float mxs[8];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+                for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i]));
+#pragma unroll
+                for (int i = 8; i < 32; ++i) mxs[i & 7] = fmaxf(mxs[i & 7], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
                 const float m_new = fmaxf(m_used, mx * p.scale_log2);
                 const bool first = t == sg.tile_begin;
                 const bool raise = __any_sync(0xffffffffu, m_new > m_used + kRaiseMaxBy);
@@ -331,13 +337,13 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                     l *= alpha;
                 }
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                float lsum = 0.f;
+                float ls[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t pk[32];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float a = ex2(fmaf(__uint_as_float(s0[2 * i]), p.scale_log2, neg_m));
                     const float b = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), p.scale_log2, neg_m));
-                    lsum += a + b;
+                    ls[i & 3] += a + b;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
                     pk[i] = *reinterpret_cast<uint32_t *>(&h2);
                 }
@@ -345,11 +351,11 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 for (int i = 0; i < 16; ++i) {
                     const float a = ex2(fmaf(__uint_as_float(s1[2 * i]), p.scale_log2, neg_m));
                     const float b = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), p.scale_log2, neg_m));
-                    lsum += a + b;
+                    ls[i & 3] += a + b;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
                     pk[16 + i] = *reinterpret_cast<uint32_t *>(&h2);
                 }
-                l += lsum;
+                l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
 
                 // the previous value product must be complete before P or O are touched
                 if (it > 0) {
