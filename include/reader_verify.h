@@ -43,6 +43,7 @@ extern "C" {
 
 #define READER_MAX_NODES 128
 #define READER_PAGE_SIZE 64
+#define READER_NOALLOC_MAX_ROWS 4096 /* batch * n_nodes limit of reader_accept_noalloc */
 
 typedef struct reader_ctx reader_ctx; /* opaque: device id, SM count, driver entry points */
 
@@ -55,7 +56,8 @@ typedef enum {
     READER_ERR_UNSUPPORTED = 5, /* shape the kernels are not built for */
     READER_ERR_TIMEOUT = 6,     /* status word: a bounded device-side wait gave up */
     READER_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed */
-    READER_ERR_BAD_PAGE = 8     /* status word: page-table entry outside [0, num_pages) */
+    READER_ERR_BAD_PAGE = 8,    /* status word: page-table entry outside [0, num_pages) */
+    READER_ERR_TOO_LARGE = 9    /* more rows than reader_accept_noalloc's built-in scratch holds */
 } reader_status;
 
 /*
@@ -177,6 +179,28 @@ reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const vo
                                const int32_t *path, const int32_t *n_acc, int32_t max_path,
                                int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out,
                                void *stream);
+
+/*
+ * reader_accept with target logits, for callers that cannot provide a workspace.  (The paper has
+ * no counterpart: this exists only because of how the library is deployed.)  Think of a serving
+ * process that gave all device memory to its own pool at start-up, or a decode loop that may not
+ * make an allocating call between steps: neither can cudaMalloc the scratch reader_accept wants.
+ * Here the per-block (maximum, index) pairs of the logits scan live in a 2 MiB array inside the
+ * library's device image instead; every GPU that loads the library holds it until the process
+ * exits.  Inputs, outputs and results are exactly those of reader_accept(logits != NULL).
+ *   - batch * n_nodes must not exceed READER_NOALLOC_MAX_ROWS, else READER_ERR_TOO_LARGE is
+ *     returned and nothing is launched.
+ *   - The call allocates nothing.  Its first use on a device looks up the array's device address
+ *     (once per device; the context's device must be current): make that first call before any
+ *     stream capture begins.
+ *   - All calls share the array and leave their pairs in it.  Nothing in it needs clearing, every
+ *     slot read is written earlier in the same call; but calls that can overlap on the GPU (two
+ *     streams, two host threads) race on it -- issue them on one stream or order them.
+ */
+reader_status reader_accept_noalloc(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens,
+                                    const float *logits, int32_t vocab, int32_t *target_ids,
+                                    int32_t max_path, int32_t *path_out, int32_t *n_acc_out,
+                                    int32_t *bonus_out, int32_t *status_out, void *stream);
 
 #ifdef __cplusplus
 }

@@ -18,12 +18,14 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libreader_verify.so")
 
-OK, ERR_INVALID_ARG, ERR_BAD_TREE, ERR_CAPACITY, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_CUDA, ERR_BAD_PAGE = range(9)
+(OK, ERR_INVALID_ARG, ERR_BAD_TREE, ERR_CAPACITY, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_TIMEOUT, ERR_CUDA, ERR_BAD_PAGE,
+ ERR_TOO_LARGE) = range(10)
+NOALLOC_MAX_ROWS = 4096
 
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
            "reader_set_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
-           "reader_kv_commit")
+           "reader_kv_commit", "reader_accept_noalloc")
 
 
 class ReaderError(RuntimeError):
@@ -74,6 +76,9 @@ def load_library() -> ctypes.CDLL:
     lib.reader_accept.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
                                   c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.reader_accept.restype = c_int32
+    lib.reader_accept_noalloc.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
+                                          c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.reader_accept_noalloc.restype = c_int32
     lib.reader_kv_commit.argtypes = [c_void_p, POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
     lib.reader_kv_commit.restype = c_int32
@@ -232,6 +237,32 @@ class Reader:
                                     _ptr(ws), ws.numel(), _ptr(status), _stream())
         if st != OK:
             raise ReaderError(st, "reader_accept")
+        return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
+
+    def accept_noalloc(self, parent: torch.Tensor, node_tokens: torch.Tensor, max_path: int, logits: torch.Tensor,
+                       target_ids: Optional[torch.Tensor] = None, outs=None):
+        """reader_accept_noalloc: acceptance from target logits without a workspace.  For hosts that
+        cannot allocate device memory when they call; the scan's scratch is a fixed 2 MiB array inside
+        the library, which limits batch * n_nodes to NOALLOC_MAX_ROWS and makes concurrent calls on
+        different streams race.  When ``target_ids`` and ``outs`` are given this wrapper allocates nothing either."""
+        _dev(parent, torch.int32, "parent"); _dev(node_tokens, torch.int32, "node_tokens")
+        _dev(logits, torch.float32, "logits")
+        B, T = parent.shape
+        dev = parent.device
+        if target_ids is None:
+            target_ids = torch.empty((B, T), dtype=torch.int32, device=dev)
+        _dev(target_ids, torch.int32, "target_ids")
+        if outs is None:
+            outs = (torch.empty((B, max_path), dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev))
+        path, n_acc, bonus, status = outs
+        tree = _Tree(B, T, parent.data_ptr(), None)
+        st = self.lib.reader_accept_noalloc(self._h, ctypes.byref(tree), _ptr(node_tokens), _ptr(logits),
+                                            logits.shape[-1], _ptr(target_ids), int(max_path), _ptr(path),
+                                            _ptr(n_acc), _ptr(bonus), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_accept_noalloc")
         return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
 
     def kv_commit(self, cache: KvCache, k_tree: torch.Tensor, v_tree: torch.Tensor, path: torch.Tensor,

@@ -3,15 +3,8 @@
 #include <new>
 
 #include "common.cuh"
-#include "verify_attn_sm100.cuh"
+#include "ctx.cuh"
 
-struct reader_ctx {
-    int device;
-    int n_sm;
-    int attn_kernel;  // 0 auto, 1 generic (CUDA cores), 2 tensor-core kernel only
-    reader::Sm100Host sm100;
-    cudaEvent_t ev_start, ev_stop;  // optional timing hooks around the main attention kernel
-};
 
 namespace {
 
@@ -105,6 +98,7 @@ const char *reader_status_string(reader_status s) {
         case READER_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case READER_ERR_CUDA: return "CUDA call failed";
         case READER_ERR_BAD_PAGE: return "page id outside the pool";
+        case READER_ERR_TOO_LARGE: return "problem larger than the built-in scratch of the allocation-free entry point";
     }
     return "unknown status";
 }
