@@ -1,15 +1,19 @@
 // Tree-masked verify attention (Sec. 3.2) on the sm_100a tensor cores.
 //
-// Two persistent CTAs per SM each walk their range of the flattened split-KV tile list.  For every unit
-// (sequence, KV head, 128 query rows) it computes S = Q K^T and O += P V with tcgen05.mma, one KV
-// tile of 64 keys (one cache page, or 64 tree nodes) at a time:
+// Two persistent CTAs per SM each walk their range of the flattened split-KV tile list.  For every
+// unit (sequence, KV head, 128 query rows) a CTA computes S = Q K^T and O += P V with tcgen05.mma,
+// one KV tile of 64 keys (one cache page, or 64 tree nodes) at a time:
 //
-//   warp 4      producer: full cache pages arrive by TMA (two 64x64 boxes per K and per V tile,
-//               128-byte swizzle) into a ring of kStages stages; the ragged last page and the
-//               tree tiles are copied with ordinary loads and zero-filled past their end, so that
-//               bytes beyond a sequence's length can never reach a product
-//   warp 5      MMA issuer: S[t+1] = Q K[t+1]^T is issued ahead of O += P[t] V[t], so the tensor
-//               pipe works on the next scores while the softmax warps are busy with this tile
+//   warp 4      producer: K tiles and V tiles travel through two separate rings of kStages
+//               slots.  Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages
+//               from the pool, tree tiles from the tree tensors.  A K slot is free again as soon
+//               as its score product has run, long before the tile's value product, so key loads
+//               run far ahead.  Bytes beyond a sequence's length or the tree's end can never
+//               reach a product: scores there are replaced by -inf, and the value product skips
+//               16-key slices past the end and zeroes the tail of the last slice in place.
+//   warp 5      MMA issuer, event driven: it issues S[i] = Q K[i]^T whenever K[i] has landed and
+//               a score buffer is free, and O += P[j] V[j] whenever P[j] and V[j] are ready; it
+//               never sits on one barrier while the other kind of work could be issued.
 //   warps 0-3   softmax: thread r owns query row r = TMEM lane r.  Scores come from TMEM, the
 //               ancestor bitmask / length mask is applied, the running maximum is raised only
 //               when it grows by more than 2^8 (the accumulator in TMEM is rescaled then),
@@ -18,8 +22,8 @@
 //               partial) at its end.
 //
 // TMEM: columns 0-127 hold two score buffers of 64 columns, columns 128.. hold O (head_dim
-// columns), all fp32, lane = query row.  Every wait on an mbarrier is bounded: after one second a
-// CTA raises the error flag in the workspace, stops waiting and runs to its end.
+// columns), all fp32, lane = query row.  Every wait on an mbarrier is bounded: after one second
+// without progress a CTA raises the error flag in the workspace, stops waiting and runs to its end.
 #include <cuda.h>
 
 #include <new>
@@ -49,16 +53,16 @@ struct Cfg {
     static constexpr int kQBytes = kTileM * D * 2;
     static constexpr int kPBytes = kTileM * kPage * 2;
     static constexpr int kTileBytes = kPage * D * 2;
-    static constexpr int kStageBytes = 2 * kTileBytes;
     static constexpr int kOffQ = 0;
     static constexpr int kOffP = kQBytes;
-    static constexpr int kOffStages = kOffP + kPBytes;
-    static constexpr int kOffBars = kOffStages + kStages * kStageBytes;
+    static constexpr int kOffK = kOffP + kPBytes;                 // ring of K tiles
+    static constexpr int kOffV = kOffK + kStages * kTileBytes;    // ring of V tiles
+    static constexpr int kOffBars = kOffV + kStages * kTileBytes;
     static constexpr int kSmemBytes = kOffBars + 256;   // + barriers; two CTAs of head_dim 128 fit one SM
 };
 
 struct Bars {
-    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
     uint64_t q_full, s_full[2], s_empty[2], p_full, pv_done;
     uint32_t tmem_base;
     int32_t abort;
@@ -81,9 +85,97 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int
     }
 }
 
+
+// Gives up after kWaitLimitNs without progress in a polling loop.
+struct Watchdog {
+    uint64_t t0 = 0;
+    bool armed = false;
+    __device__ __forceinline__ void progress() { armed = false; }
+    __device__ __forceinline__ bool expired(volatile int32_t *abort_s, int32_t *error_flag) {
+        if (*abort_s) return true;
+        if (!armed) {
+            armed = true;
+            t0 = globaltimer_ns();
+            return false;
+        }
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *abort_s = 1;
+            atomicExch(error_flag, (int32_t)READER_ERR_TIMEOUT);
+            return true;
+        }
+        return false;
+    }
+};
+
+// Warp-uniform, non-blocking test of an mbarrier phase (true only once every lane has seen it).
+__device__ __forceinline__ bool ready(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_test_wait(bar, parity));
+}
+
+// Walks the tiles of a CTA's range in order; the producer keeps one cursor for keys and one for
+// values.  Page ids are fetched 32 at a time (one per lane) and handed out by shuffle.
+struct TileCursor {
+    int w, w_end;       // flat position of the next segment
+    Segment sg;
+    int L;              // committed length of sg.b
+    int t;              // current tile within the unit
+    int it;             // tiles handed out so far
+    int cache_t0, cache_page;
+    bool active;
+
+    __device__ __forceinline__ void refill(const AttnParams &p, int lane) {
+        cache_t0 = t;
+        const int tt = t + lane;
+        cache_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
+    }
+    __device__ __forceinline__ void next_segment(const AttnParams &p, int cta, int lane) {
+        active = w < w_end;
+        if (!active) return;
+        sg = segment_at(p.sched, p.B, cta, w, w_end);
+        w += sg.tile_end - sg.tile_begin;
+        L = p.seq_lens[sg.b];
+        t = sg.tile_begin;
+        refill(p, lane);
+    }
+    __device__ __forceinline__ void init(const AttnParams &p, int cta, int lane, int w_begin, int w_end_) {
+        w = w_begin; w_end = w_end_; it = 0;
+        next_segment(p, cta, lane);
+    }
+    __device__ __forceinline__ int page() const { return __shfl_sync(0xffffffffu, cache_page, t - cache_t0); }
+    __device__ __forceinline__ void advance(const AttnParams &p, int cta, int lane) {
+        ++t; ++it;
+        if (t == sg.tile_end) next_segment(p, cta, lane);
+        else if (t - cache_t0 == 32) refill(p, lane);
+    }
+};
+
+// One K or V tile into its ring slot, always by TMA: a cache page comes whole from the pool (the
+// page exists in full even when the sequence ends inside it), a tree tile comes as 64 node rows of
+// one KV head from the tree tensor (rows past the tensor's end read as zero).  Rows past the
+// valid count may therefore hold anything; the score side masks them by selection and the value
+// side never multiplies them (see the MMA issuer).  Called by the whole producer warp.
+template <int D>
+__device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor &c, const CUtensorMap *pool_map,
+                                          const CUtensorMap *tree_map, uint32_t dst, uint32_t full, int lane) {
+    using C = Cfg<D>;
+    const int page = c.page();
+    if (lane != 0) return;
+    mbar_arrive_expect_tx(full, C::kTileBytes);
+    if (c.t < c.sg.npages) {
+        const int row = (page * p.Hkv + c.sg.h) * kPage;
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf) tma_load_2d(dst + hf * C::kHalfRowsKV, pool_map, full, hf * 64, row);
+    } else {
+        const int node0 = c.sg.b * p.T + (c.t - c.sg.npages) * kPage;
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf) tma_load_3d(dst + hf * C::kHalfRowsKV, tree_map, full, hf * 64, c.sg.h, node0);
+    }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 2)
-attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
+attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
+                  const __grid_constant__ CUtensorMap ktmap, const __grid_constant__ CUtensorMap vtmap) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t base = smem_u32(smem);
@@ -97,13 +189,15 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
 
-    const uint32_t sQ = base + C::kOffQ, sP = base + C::kOffP, sStages = base + C::kOffStages;
+    const uint32_t sQ = base + C::kOffQ, sP = base + C::kOffP, sK = base + C::kOffK, sV = base + C::kOffV;
     auto bar = [&](const uint64_t *b) { return smem_u32(b); };
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar(&bars->kv_full[s]), 1);
-            mbar_init(bar(&bars->kv_empty[s]), 1);
+            mbar_init(bar(&bars->k_full[s]), 1);
+            mbar_init(bar(&bars->k_empty[s]), 1);
+            mbar_init(bar(&bars->v_full[s]), 1);
+            mbar_init(bar(&bars->v_empty[s]), 1);
         }
         mbar_init(bar(&bars->q_full), kTileM);
         for (int s = 0; s < 2; ++s) {
@@ -134,130 +228,124 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         if (lane == 0) {
             prefetch_tensormap(&kmap);
             prefetch_tensormap(&vmap);
+            prefetch_tensormap(&ktmap);
+            prefetch_tensormap(&vtmap);
         }
-        int it = 0;
-        int w = w_begin;
-        while (w < w_end) {
-            const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
-            w += sg.tile_end - sg.tile_begin;
-            const int L = p.seq_lens[sg.b];
-            for (int t0 = sg.tile_begin; t0 < sg.tile_end; t0 += 32) {
-                const int tt = t0 + lane;
-                const int my_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
-                const int n = min(32, sg.tile_end - t0);
-                for (int i = 0; i < n; ++i, ++it) {
-                    const int t = t0 + i;
-                    const int page = __shfl_sync(0xffffffffu, my_page, i);
-                    const int stage = it % kStages;
-                    wait(bar(&bars->kv_empty[stage]), ((it / kStages) & 1) ^ 1, abort_s, p.error_flag);
-                    const uint32_t kdst = sStages + stage * C::kStageBytes, vdst = kdst + C::kTileBytes;
-                    const uint32_t full = bar(&bars->kv_full[stage]);
-                    const bool whole_page = t < sg.npages && L - t * kPage >= kPage;
-                    if (whole_page) {
-                        if (lane == 0) {
-                            mbar_arrive_expect_tx(full, C::kStageBytes);
-                            const int row = (page * p.Hkv + sg.h) * kPage;
-#pragma unroll
-                            for (int hf = 0; hf < C::kHalves; ++hf) {
-                                tma_load_2d(kdst + hf * C::kHalfRowsKV, &kmap, full, hf * 64, row);
-                                tma_load_2d(vdst + hf * C::kHalfRowsKV, &vmap, full, hf * 64, row);
-                            }
-                        }
-                    } else {
-                        const __nv_bfloat16 *ksrc, *vsrc;
-                        size_t stride;
-                        int valid;
-                        if (t < sg.npages) {
-                            const size_t at = ((size_t)page * p.Hkv + sg.h) * kPage * D;
-                            ksrc = p.k_pool + at; vsrc = p.v_pool + at;
-                            stride = D;
-                            valid = L - t * kPage;
-                        } else {
-                            const int kt = t - sg.npages;
-                            const size_t at = (((size_t)sg.b * p.T + kt * kPage) * p.Hkv + sg.h) * D;
-                            ksrc = p.k_tree + at; vsrc = p.v_tree + at;
-                            stride = (size_t)p.Hkv * D;
-                            valid = min(kPage, p.T - kt * kPage);
-                        }
-                        constexpr int kChunks = D / 8;
-#pragma unroll 4
-                        for (int c = lane; c < kPage * kChunks; c += 32) {
-                            const int rr = c / kChunks, cc = c % kChunks;
-                            uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-                            if (rr < valid) {
-                                kv = *reinterpret_cast<const uint4 *>(ksrc + rr * stride + cc * 8);
-                                vv = *reinterpret_cast<const uint4 *>(vsrc + rr * stride + cc * 8);
-                            }
-                            const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(kdst + off), "r"(kv.x), "r"(kv.y), "r"(kv.z), "r"(kv.w) : "memory");
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(vdst + off), "r"(vv.x), "r"(vv.y), "r"(vv.z), "r"(vv.w) : "memory");
-                        }
-                        fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(full);
-                    }
+        TileCursor kc, vc;
+        kc.init(p, cta, lane, w_begin, w_end);
+        vc.init(p, cta, lane, w_begin, w_end);
+        Watchdog dog;
+        while (kc.active || vc.active) {
+            bool moved = false;
+            if (kc.active) {
+                const int stage = kc.it % kStages;
+                if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStages) & 1) ^ 1)) {
+                    load_tile<D>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane);
+                    __syncwarp();
+                    kc.advance(p, cta, lane);
+                    moved = true;
                 }
             }
+            if (vc.active) {
+                const int stage = vc.it % kStages;
+                if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStages) & 1) ^ 1)) {
+                    load_tile<D>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane);
+                    __syncwarp();
+                    vc.advance(p, cta, lane);
+                    moved = true;
+                }
+            }
+            if (moved) dog.progress();
+            else if (dog.expired(abort_s, p.error_flag)) break;
         }
         // a CTA that gave up must not exit under its own copies: let the last ones land (bounded)
         if (*abort_s) {
             const uint64_t t0 = globaltimer_ns();
-            for (int i = max(0, it - kStages); i < it; ++i)
-                while (!mbar_try_wait(bar(&bars->kv_full[i % kStages]), (i / kStages) & 1) &&
-                       globaltimer_ns() - t0 < 20000000ull) {
+            for (int i = max(0, kc.it - kStages); i < kc.it; ++i)
+                while (!mbar_try_wait(bar(&bars->k_full[i % kStages]), (i / kStages) & 1) && globaltimer_ns() - t0 < 20000000ull) {
+                }
+            for (int i = max(0, vc.it - kStages); i < vc.it; ++i)
+                while (!mbar_try_wait(bar(&bars->v_full[i % kStages]), (i / kStages) & 1) && globaltimer_ns() - t0 < 20000000ull) {
                 }
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
         constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kPage, false, false);
         constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, false, true);
-        auto issue_qk = [&](int i) {
-            const int stage = i % kStages, buf = i & 1;
-            wait(bar(&bars->kv_full[stage]), (i / kStages) & 1, abort_s, p.error_flag);
-            wait(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1, abort_s, p.error_flag);
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t kbase = sStages + stage * C::kStageBytes;
-#pragma unroll
-                for (int hf = 0; hf < C::kHalves; ++hf)
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t a = smem_desc_sw128(sQ + hf * C::kHalfRowsQ + kk * 32, 16, 1024);
-                        const uint64_t b = smem_desc_sw128(kbase + hf * C::kHalfRowsKV + kk * 32, 16, 1024);
-                        mma_bf16_ss(tmem + buf * kPage, a, b, kIdescQK, (hf | kk) != 0);
-                    }
-                mma_commit(bar(&bars->s_full[buf]));
-            }
-            __syncwarp();
-        };
-        int it = 0, seg = 0;
+        int it0 = 0, seg = 0;
         int w = w_begin;
-        while (w < w_end) {
+        Watchdog dog;
+        while (w < w_end && !*abort_s) {
             const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
             const int n = sg.tile_end - sg.tile_begin;
             w += n;
+            const int L = p.seq_lens[sg.b];
             wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
             tc_fence_after();
-            issue_qk(it);
-            for (int t = 0; t < n; ++t) {
-                if (t + 1 < n) issue_qk(it + t + 1);
-                wait(bar(&bars->p_full), (it + t) & 1, abort_s, p.error_flag);
-                tc_fence_after();
-                if (lane == 0) {
-                    const int stage = (it + t) % kStages;
-                    const uint32_t vbase = sStages + stage * C::kStageBytes + C::kTileBytes;
+            int next_qk = 0, next_pv = 0;
+            while (next_pv < n) {
+                bool moved = false;
+                if (next_qk < n) {
+                    const int i = it0 + next_qk, stage = i % kStages, buf = i & 1;
+                    if (ready(bar(&bars->k_full[stage]), (i / kStages) & 1) &&
+                        ready(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1)) {
+                        tc_fence_after();
+                        if (lane == 0) {
+                            const uint32_t kbase = sK + stage * C::kTileBytes;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t a = smem_desc_sw128(sP + kk * 32, 16, 1024);
-                        const uint64_t b = smem_desc_sw128(vbase + kk * 2048, C::kHalfRowsKV, 1024);
-                        mma_bf16_ss(tmem + kTmemO, a, b, kIdescPV, (t | kk) != 0);
+                            for (int hf = 0; hf < C::kHalves; ++hf)
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const uint64_t a = smem_desc_sw128(sQ + hf * C::kHalfRowsQ + kk * 32, 16, 1024);
+                                    const uint64_t b = smem_desc_sw128(kbase + hf * C::kHalfRowsKV + kk * 32, 16, 1024);
+                                    mma_bf16_ss(tmem + buf * kPage, a, b, kIdescQK, (hf | kk) != 0);
+                                }
+                            mma_commit(bar(&bars->k_empty[stage]));
+                            mma_commit(bar(&bars->s_full[buf]));
+                        }
+                        __syncwarp();
+                        ++next_qk;
+                        moved = true;
                     }
-                    mma_commit(bar(&bars->kv_empty[stage]));
-                    mma_commit(bar(&bars->pv_done));
                 }
-                __syncwarp();
+                if (next_pv < next_qk) {
+                    const int i = it0 + next_pv, stage = i % kStages;
+                    if (ready(bar(&bars->p_full), i & 1) && ready(bar(&bars->v_full[stage]), (i / kStages) & 1)) {
+                        tc_fence_after();
+                        const uint32_t vbase = sV + stage * C::kTileBytes;
+                        // keys past the end of the sequence / tree: whole 16-key slices are not
+                        // multiplied at all, the rest of the last slice is zeroed in place
+                        const int t = sg.tile_begin + next_pv;
+                        const int valid = t < sg.npages ? min(kPage, L - t * kPage) : min(kPage, p.T - (t - sg.npages) * kPage);
+                        const int slices = (valid + 15) >> 4;
+                        if (valid & 15) {
+                            constexpr int kChunks = D / 8;
+                            for (int idx = lane; idx < (slices * 16 - valid) * kChunks; idx += 32) {
+                                const int rr = valid + idx / kChunks, cc = idx % kChunks;
+                                const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
+                            }
+                            fence_proxy_async();
+                            __syncwarp();
+                        }
+                        if (lane == 0) {
+                            for (int kk = 0; kk < slices; ++kk) {
+                                const uint64_t a = smem_desc_sw128(sP + kk * 32, 16, 1024);
+                                const uint64_t b = smem_desc_sw128(vbase + kk * 2048, C::kHalfRowsKV, 1024);
+                                mma_bf16_ss(tmem + kTmemO, a, b, kIdescPV, (next_pv | kk) != 0);
+                            }
+                            mma_commit(bar(&bars->v_empty[stage]));
+                            mma_commit(bar(&bars->pv_done));
+                        }
+                        __syncwarp();
+                        ++next_pv;
+                        moved = true;
+                    }
+                }
+                if (moved) dog.progress();
+                else if (dog.expired(abort_s, p.error_flag)) break;
             }
-            it += n;
+            it0 += n;
             ++seg;
         }
     } else {
@@ -454,13 +542,28 @@ bool encode_pool_map(void *fn, CUtensorMap *map, const void *pool, int64_t rows,
                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D view of a tree tensor [B*T nodes][Hkv][D]: box = 64 columns x 1 head x 64 nodes.
+bool encode_tree_map(void *fn, CUtensorMap *map, const void *tree, int64_t nodes, int Hkv, int D) {
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)nodes};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kPage};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return reinterpret_cast<EncodeTiledFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(tree), dims,
+                                               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 struct Sm100Maps {
     const void *k_pool = nullptr, *v_pool = nullptr;
     int64_t rows = -1;
     int D = 0;
-    alignas(64) CUtensorMap kmap, vmap;
+    const void *k_tree = nullptr, *v_tree = nullptr;
+    int64_t nodes = -1;
+    int tree_heads = 0, tree_D = 0;
+    alignas(64) CUtensorMap kmap, vmap, ktmap, vtmap;
 };
 
 reader_status sm100_host_init(Sm100Host *h, int device) {
@@ -518,10 +621,19 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_
         }
         m->k_pool = cache.k_pool; m->v_pool = cache.v_pool; m->rows = rows; m->D = p.D;
     }
+    const int64_t nodes = (int64_t)p.B * p.T;
+    if (m->k_tree != p.k_tree || m->v_tree != p.v_tree || m->nodes != nodes || m->tree_heads != p.Hkv || m->tree_D != p.D) {
+        if (!encode_tree_map(h->encode_tiled, &m->ktmap, p.k_tree, nodes, p.Hkv, p.D) ||
+            !encode_tree_map(h->encode_tiled, &m->vtmap, p.v_tree, nodes, p.Hkv, p.D)) {
+            m->nodes = -1;
+            return READER_ERR_CUDA;
+        }
+        m->k_tree = p.k_tree; m->v_tree = p.v_tree; m->nodes = nodes; m->tree_heads = p.Hkv; m->tree_D = p.D;
+    }
     if (p.D == 128)
-        attn_sm100_kernel<128><<<p.sched.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p, m->kmap, m->vmap);
+        attn_sm100_kernel<128><<<p.sched.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap);
     else
-        attn_sm100_kernel<64><<<p.sched.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p, m->kmap, m->vmap);
+        attn_sm100_kernel<64><<<p.sched.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap);
     return READER_OK;
 }
 
