@@ -72,6 +72,32 @@ __device__ __forceinline__ Segment segment_at(const Sched &s, int B, int cta, in
     return g;
 }
 
+// Same result as segment_at, for a whole warp calling together: the sequence is found with one
+// round of parallel loads per 32 sequences instead of a chain of dependent ones.
+__device__ __forceinline__ Segment segment_at_warp(const Sched &s, int B, int cta, int w, int range_end, int lane) {
+    int b = 0;
+    for (int base = 0; base < B; base += 32) {
+        const int i = base + lane;
+        const unsigned le = __ballot_sync(0xffffffffu, i < B && s.seq_tile_start[i] <= w);
+        if (le) b = base + 31 - __clz(le);   // the starts never decrease: the set bits are a prefix
+        if (le != 0xffffffffu) break;
+    }
+    Segment g;
+    g.b = b;
+    g.ntiles = s.seq_ntiles[b];
+    g.npages = s.seq_npages[b];
+    int local = w - s.seq_tile_start[b];
+    int unit = local / g.ntiles;
+    g.tile_begin = local - unit * g.ntiles;
+    g.h = unit / s.n_mtiles;
+    g.mt = unit - g.h * s.n_mtiles;
+    int left = range_end - w;
+    g.tile_end = min(g.ntiles, g.tile_begin + left);
+    g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
+    g.slot = 2 * cta + (g.tile_begin == 0 ? 1 : 0);
+    return g;
+}
+
 // CTA whose range contains flat tile w.
 __device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
     int c = (int)(((int64_t)w * n_ctas) / W);

@@ -18,8 +18,9 @@
 //               ancestor bitmask / length mask is applied, the running maximum is raised only
 //               when it grows by more than 2^8 (the accumulator in TMEM is rescaled then),
 //               probabilities go to shared memory as the bf16 A operand of the value product.
-//               The same threads stage Q at the start of a segment and write O (or an (m, l, O)
-//               partial) at its end.
+//               The same threads write O (or an (m, l, O) partial) at the end of a segment.
+// The 128 query rows of a unit (node j, group member g -> row j*G+g) come in by one 4-D TMA box per
+// 64 columns, issued by the producer as soon as the previous segment's last score product is done.
 //
 // TMEM: columns 0-127 hold two score buffers of 64 columns, columns 128.. hold O (head_dim
 // columns), all fp32, lane = query row.  Every wait on an mbarrier is bounded: after one second
@@ -63,7 +64,7 @@ struct Cfg {
 
 struct Bars {
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-    uint64_t q_full, s_full[2], s_empty[2], p_full, pv_done;
+    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full, pv_done;
     uint32_t tmem_base;
     int32_t abort;
 };
@@ -131,7 +132,7 @@ struct TileCursor {
     __device__ __forceinline__ void next_segment(const AttnParams &p, int cta, int lane) {
         active = w < w_end;
         if (!active) return;
-        sg = segment_at(p.sched, p.B, cta, w, w_end);
+        sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
         w += sg.tile_end - sg.tile_begin;
         L = p.seq_lens[sg.b];
         t = sg.tile_begin;
@@ -175,7 +176,8 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
-                  const __grid_constant__ CUtensorMap ktmap, const __grid_constant__ CUtensorMap vtmap) {
+                  const __grid_constant__ CUtensorMap ktmap, const __grid_constant__ CUtensorMap vtmap,
+                  const __grid_constant__ CUtensorMap qmap) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t base = smem_u32(smem);
@@ -199,7 +201,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             mbar_init(bar(&bars->v_full[s]), 1);
             mbar_init(bar(&bars->v_empty[s]), 1);
         }
-        mbar_init(bar(&bars->q_full), kTileM);
+        mbar_init(bar(&bars->q_full), 1);
+        mbar_init(bar(&bars->q_empty), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(&bars->s_full[s]), 1);
             mbar_init(bar(&bars->s_empty[s]), kTileM);
@@ -230,13 +233,32 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             prefetch_tensormap(&vmap);
             prefetch_tensormap(&ktmap);
             prefetch_tensormap(&vtmap);
+            prefetch_tensormap(&qmap);
         }
         TileCursor kc, vc;
         kc.init(p, cta, lane, w_begin, w_end);
         vc.init(p, cta, lane, w_begin, w_end);
+        // the query tile of the next segment goes in as soon as the last score product of the
+        // current one has retired (Q is single-buffered)
+        int q_w = w_begin, q_seg = 0;
+        const int rows_per_node_tile = kTileM / p.G;
         Watchdog dog;
-        while (kc.active || vc.active) {
+        while (kc.active || vc.active || q_w < w_end) {
             bool moved = false;
+            if (q_w < w_end && ready(bar(&bars->q_empty), (q_seg & 1) ^ 1)) {
+                const Segment sg = segment_at_warp(p.sched, p.B, cta, q_w, w_end, lane);
+                q_w += sg.tile_end - sg.tile_begin;
+                if (lane == 0) {
+                    const uint32_t full = bar(&bars->q_full);
+                    mbar_arrive_expect_tx(full, C::kQBytes);
+#pragma unroll
+                    for (int hf = 0; hf < C::kHalves; ++hf)
+                        tma_load_4d(sQ + hf * C::kHalfRowsQ, &qmap, full, hf * 64, sg.h * p.G, sg.mt * rows_per_node_tile, sg.b);
+                }
+                __syncwarp();
+                ++q_seg;
+                moved = true;
+            }
             if (kc.active) {
                 const int stage = kc.it % kStages;
                 if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStages) & 1) ^ 1)) {
@@ -272,11 +294,15 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         // ------------------------------------------------------------------ MMA issuer
         constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kPage, false, false);
         constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, false, true);
+        // descriptors differ only in their start-address field (bytes >> 4), so each operand's
+        // descriptor is one addition away from a base built once
+        const uint64_t descQ = smem_desc_sw128(sQ, 16, 1024), descK = smem_desc_sw128(sK, 16, 1024);
+        const uint64_t descP = smem_desc_sw128(sP, 16, 1024), descV = smem_desc_sw128(sV, C::kHalfRowsKV, 1024);
         int it0 = 0, seg = 0;
         int w = w_begin;
         Watchdog dog;
         while (w < w_end && !*abort_s) {
-            const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
+            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += n;
             const int L = p.seq_lens[sg.b];
@@ -291,17 +317,16 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                         ready(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1)) {
                         tc_fence_after();
                         if (lane == 0) {
-                            const uint32_t kbase = sK + stage * C::kTileBytes;
+                            const uint64_t kd = descK + (uint64_t)((stage * C::kTileBytes) >> 4);
 #pragma unroll
                             for (int hf = 0; hf < C::kHalves; ++hf)
 #pragma unroll
-                                for (int kk = 0; kk < 4; ++kk) {
-                                    const uint64_t a = smem_desc_sw128(sQ + hf * C::kHalfRowsQ + kk * 32, 16, 1024);
-                                    const uint64_t b = smem_desc_sw128(kbase + hf * C::kHalfRowsKV + kk * 32, 16, 1024);
-                                    mma_bf16_ss(tmem + buf * kPage, a, b, kIdescQK, (hf | kk) != 0);
-                                }
+                                for (int kk = 0; kk < 4; ++kk)
+                                    mma_bf16_ss(tmem + buf * kPage, descQ + (uint64_t)((hf * C::kHalfRowsQ + kk * 32) >> 4),
+                                                kd + (uint64_t)((hf * C::kHalfRowsKV + kk * 32) >> 4), kIdescQK, (hf | kk) != 0);
                             mma_commit(bar(&bars->k_empty[stage]));
                             mma_commit(bar(&bars->s_full[buf]));
+                            if (next_qk == n - 1) mma_commit(bar(&bars->q_empty));
                         }
                         __syncwarp();
                         ++next_qk;
@@ -329,11 +354,12 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                             __syncwarp();
                         }
                         if (lane == 0) {
-                            for (int kk = 0; kk < slices; ++kk) {
-                                const uint64_t a = smem_desc_sw128(sP + kk * 32, 16, 1024);
-                                const uint64_t b = smem_desc_sw128(vbase + kk * 2048, C::kHalfRowsKV, 1024);
-                                mma_bf16_ss(tmem + kTmemO, a, b, kIdescPV, (next_pv | kk) != 0);
-                            }
+                            const uint64_t vd = descV + (uint64_t)((stage * C::kTileBytes) >> 4);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)
+                                if (kk < slices)
+                                    mma_bf16_ss(tmem + kTmemO, descP + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4),
+                                                kIdescPV, (next_pv | kk) != 0);
                             mma_commit(bar(&bars->v_empty[stage]));
                             mma_commit(bar(&bars->pv_done));
                         }
@@ -354,7 +380,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int it = 0;
         int w = w_begin;
         while (w < w_end) {
-            const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
+            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
             w += sg.tile_end - sg.tile_begin;
             const int L = p.seq_lens[sg.b];
             const int grow = sg.mt * kTileM + tid;
@@ -363,18 +389,6 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             const int hq = sg.h * p.G + (row_ok ? grow % p.G : 0);
             const size_t qrow = (((size_t)sg.b * p.T + j) * p.Hq + hq) * D;
 
-            // stage this thread's query row (128-byte swizzle, zero for padding rows)
-            {
-                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + qrow);
-#pragma unroll
-                for (int c = 0; c < D / 8; ++c) {
-                    const uint4 v = row_ok ? src[c] : make_uint4(0, 0, 0, 0);
-                    const uint32_t off = (c >> 3) * C::kHalfRowsQ + tid * 128 + (((c & 7) ^ (tid & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQ + off), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-                }
-                fence_proxy_async();
-                mbar_arrive(bar(&bars->q_full));
-            }
             uint64_t anc_lo = 0, anc_hi = 0;
             if (row_ok) {
                 anc_lo = p.anc[((size_t)sg.b * p.T + j) * 2 + 0];
@@ -554,6 +568,19 @@ bool encode_tree_map(void *fn, CUtensorMap *map, const void *tree, int64_t nodes
                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 4-D view of q [B][T][Hq][D]: box = 64 columns x G heads x 128/G nodes x 1 sequence, which lands in
+// shared memory as 128 rows ordered (node, group member).
+bool encode_q_map(void *fn, CUtensorMap *map, const void *q, int B, int T, int Hq, int G, int D) {
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)Hq * D * 2, (cuuint64_t)T * Hq * D * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)(kTileM / G), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return reinterpret_cast<EncodeTiledFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(q), dims,
+                                               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 struct Sm100Maps {
@@ -563,7 +590,9 @@ struct Sm100Maps {
     const void *k_tree = nullptr, *v_tree = nullptr;
     int64_t nodes = -1;
     int tree_heads = 0, tree_D = 0;
-    alignas(64) CUtensorMap kmap, vmap, ktmap, vtmap;
+    const void *q = nullptr;
+    int qB = -1, qT = 0, qHq = 0, qG = 0, qD = 0;
+    alignas(64) CUtensorMap kmap, vmap, ktmap, vtmap, qmap;
 };
 
 reader_status sm100_host_init(Sm100Host *h, int device) {
@@ -599,6 +628,7 @@ bool sm100_supports(const Sm100Host *h, const AttnParams &p, float softmax_scale
     if (!h->ready) return false;
     if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return false;   // the row maximum is taken before scaling
     const int64_t rows = (int64_t)p.num_pages * p.Hkv * kPage;
+    if (p.G > kTileM || kTileM % p.G != 0) return false;   // a query tile is a box of whole nodes
     return (p.D == 64 || p.D == 128) && rows >= 1 && rows < ((int64_t)1 << 31);
 }
 
@@ -630,10 +660,17 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_
         }
         m->k_tree = p.k_tree; m->v_tree = p.v_tree; m->nodes = nodes; m->tree_heads = p.Hkv; m->tree_D = p.D;
     }
+    if (m->q != p.q || m->qB != p.B || m->qT != p.T || m->qHq != p.Hq || m->qG != p.G || m->qD != p.D) {
+        if (!encode_q_map(h->encode_tiled, &m->qmap, p.q, p.B, p.T, p.Hq, p.G, p.D)) {
+            m->qB = -1;
+            return READER_ERR_CUDA;
+        }
+        m->q = p.q; m->qB = p.B; m->qT = p.T; m->qHq = p.Hq; m->qG = p.G; m->qD = p.D;
+    }
     if (p.D == 128)
-        attn_sm100_kernel<128><<<p.sched.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap);
+        attn_sm100_kernel<128><<<p.sched.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
     else
-        attn_sm100_kernel<64><<<p.sched.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap);
+        attn_sm100_kernel<64><<<p.sched.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
     return READER_OK;
 }
 
