@@ -17,7 +17,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct WsLayout {
-    size_t error_flag, seq_tile_start, seq_ntiles, seq_npages, anc, partial_ml, partial_o, amax_val, amax_idx, total;
+    size_t error_flag, seq_tile_start, seq_ntiles, seq_npages, anc, split_desc, partial_ml, partial_o, amax_val, amax_idx, total;
 };
 
 inline int max_ctas(const reader_ctx *ctx) { return 2 * ctx->n_sm; }
@@ -32,6 +32,7 @@ WsLayout ws_layout(const reader_ctx *ctx, int B, int T, int D) {
     w.seq_ntiles = take(sizeof(int32_t) * (size_t)B);
     w.seq_npages = take(sizeof(int32_t) * (size_t)B);
     w.anc = take(sizeof(uint64_t) * 2 * (size_t)B * T);
+    w.split_desc = take(sizeof(SplitDesc) * (size_t)max_ctas(ctx));
     w.partial_ml = take(sizeof(float) * 2 * slots * kTileM);
     w.partial_o = take(sizeof(float) * slots * kTileM * (size_t)D);
     w.amax_val = take(sizeof(float) * (size_t)B * T * kMaxSplits);
@@ -176,6 +177,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.lse = lse_out;
     p.partial_o = reinterpret_cast<float *>(ws + w.partial_o);
     p.partial_ml = reinterpret_cast<float *>(ws + w.partial_ml);
+    p.split_desc = reinterpret_cast<SplitDesc *>(ws + w.split_desc);
     p.status = status_out;
     p.error_flag = reinterpret_cast<int32_t *>(ws + w.error_flag);
     p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = G;
@@ -196,7 +198,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     launch_prepare(*cache, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
                    tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
                    reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
-                   reinterpret_cast<int32_t *>(ws + w.seq_npages), status_out, p.error_flag, st);
+                   reinterpret_cast<int32_t *>(ws + w.seq_npages), status_out, p.error_flag, p.out, p.lse, Hq, D, st);
     if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
     if (use_tc) {
         if (reader_status s = launch_attn_sm100(&ctx->sm100, p, *cache, st)) return s;

@@ -1,87 +1,118 @@
 // Split-KV combine: merges the (m, l, O) partials of every unit that was cut across CTA ranges,
 //   m* = max_s m_s,  l* = sum_s l_s 2^(m_s - m*),  O = sum_s O_s 2^(m_s - m*) / l*,
 // rounds to bf16 and writes lse = ln 2 * (m* + log2 l*).  Units written directly by the attention
-// kernel are left alone; rows of sequences with a non-zero status are zeroed, and so is every row when the
-// attention kernel raised the error flag (each status word then carries that code).
+// kernel are left alone.
+//
+// The work is found without searching: the attention CTA that started a cut unit left a descriptor
+// (unit, last CTA) in the workspace, so block c reads descriptor c and merges the unit's 128
+// rows, 8 per warp in batches of 2 with the loads of a batch all in flight together.  If the
+// attention kernel raised the error flag (a bounded wait gave up), no row of the call can be
+// trusted: everything is zeroed and every status word gets the code.
 #include "common.cuh"
 
 namespace reader {
 
-__global__ void __launch_bounds__(128) combine_kernel(const AttnParams p) {
-    const int unit_global = blockIdx.x;
-    const int ups = p.sched.units_per_seq;
-    const int b = unit_global / ups;
-    const int unit = unit_global - b * ups;
-    const int h = unit / p.sched.n_mtiles;
-    const int mt = unit - h * p.sched.n_mtiles;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = blockIdx.y * 4 + warp;   // one warp per query row: the merge is latency-bound, so spread it wide
-    const int D = p.D;
-    const int nt = p.sched.seq_ntiles[b];
-    const int rows = min(kTileM, p.T * p.G - mt * kTileM);
+constexpr int kCombineWarps = 16;                       // one block per attention CTA
+constexpr int kRowsPerWarp = kTileM / kCombineWarps;    // 8 rows, merged in batches of kBatch
+constexpr int kBatch = 2;
 
-    const int err = *p.error_flag;   // a bounded wait gave up somewhere: no row of this call can be trusted
-    if (err != 0 && unit == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.status[b] = err;
-    if (nt == 0 || err != 0) {
-        if (row < rows) {
-            const int grow = mt * kTileM + row;
-            const int j = grow / p.G, hq = h * p.G + grow % p.G;
-            __nv_bfloat16 *dst = p.out + (((size_t)b * p.T + j) * p.Hq + hq) * D;
-            if (lane * 4 < D) *reinterpret_cast<uint2 *>(dst + lane * 4) = make_uint2(0, 0);
-            if (p.lse && lane == 0) p.lse[((size_t)b * p.T + j) * p.Hq + hq] = 0.f;
-        }
+__global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const AttnParams p) {
+    const int c0 = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int D = p.D;
+    const int err = *p.error_flag;
+    const SplitDesc d = p.split_desc[c0];
+    const int W = p.sched.seq_tile_start[p.B];
+
+    if (err != 0) {
+        const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+        const size_t me = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+        uint4 *o = reinterpret_cast<uint4 *>(p.out);
+        for (size_t i = me; i < (size_t)p.B * p.T * p.Hq * D / 8; i += nthreads) o[i] = make_uint4(0, 0, 0, 0);
+        if (p.lse)
+            for (size_t i = me; i < (size_t)p.B * p.T * p.Hq; i += nthreads) p.lse[i] = 0.f;
+        for (size_t i = me; i < (size_t)p.B; i += nthreads) p.status[i] = err;
         return;
     }
-    const int W = p.sched.seq_tile_start[p.B];
-    const int u0 = p.sched.seq_tile_start[b] + unit * nt;
-    const int c_first = cta_of_tile(u0, p.sched.n_ctas, W);
-    const int c_last = cta_of_tile(u0 + nt - 1, p.sched.n_ctas, W);
-    if (c_first == c_last || row >= rows) return;
+    if (d.b < 0) return;
+    const int rows = min(kTileM, p.T * p.G - d.mt * kTileM);
+    const bool has_cols = lane * 4 < D;
+    const bool all_live = W >= p.sched.n_ctas;   // with fewer tiles than CTAs some ranges are empty
 
-    {
-        const int r = row;
-        float mstar = -INFINITY;
-        for (int c = c_first; c <= c_last; ++c) {
-            if (range_begin(c + 1, p.sched.n_ctas, W) == range_begin(c, p.sched.n_ctas, W)) continue;  // empty range: wrote nothing
-            const int slot = c == c_first ? 2 * c + 1 : 2 * c;
-            mstar = fmaxf(mstar, p.partial_ml[((size_t)slot * kTileM + r) * 2]);
+    for (int rb = 0; rb < kRowsPerWarp; rb += kBatch) {
+        const int r0 = warp * kRowsPerWarp + rb;
+        if (r0 >= rows) break;
+        float mstar[kBatch], lstar[kBatch];
+        float4 acc[kBatch];
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            mstar[q] = -INFINITY; lstar[q] = 0.f;
+            acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float lstar = 0.f;
-        for (int c = c_first; c <= c_last; ++c) {
-            if (range_begin(c + 1, p.sched.n_ctas, W) == range_begin(c, p.sched.n_ctas, W)) continue;
-            const int slot = c == c_first ? 2 * c + 1 : 2 * c;
-            const float2 ml = *reinterpret_cast<const float2 *>(p.partial_ml + ((size_t)slot * kTileM + r) * 2);
-            const float wgt = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mstar);
-            lstar += ml.y * wgt;
-            if (lane * 4 < D) {
-                const float4 o = *reinterpret_cast<const float4 *>(p.partial_o + ((size_t)slot * kTileM + r) * D + lane * 4);
-                acc.x = fmaf(o.x, wgt, acc.x);
-                acc.y = fmaf(o.y, wgt, acc.y);
-                acc.z = fmaf(o.z, wgt, acc.z);
-                acc.w = fmaf(o.w, wgt, acc.w);
+        // online merge over the CTAs c0 .. c_last, two slots x kBatch rows per round of loads
+        for (int cb = c0; cb <= d.c_last; cb += 2) {
+            float2 ml[2][kBatch];
+            float4 o[2][kBatch];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int c = cb + k;
+                // a CTA with an empty range wrote nothing
+                const bool live = c <= d.c_last && (all_live || range_begin(c + 1, p.sched.n_ctas, W) != range_begin(c, p.sched.n_ctas, W));
+                const int slot = c == c0 ? 2 * c + 1 : 2 * c;
+#pragma unroll
+                for (int q = 0; q < kBatch; ++q) {
+                    const int r = min(r0 + q, kTileM - 1);
+                    ml[k][q] = make_float2(-INFINITY, 0.f);
+                    o[k][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (live) {
+                        ml[k][q] = *reinterpret_cast<const float2 *>(p.partial_ml + ((size_t)slot * kTileM + r) * 2);
+                        if (has_cols) o[k][q] = *reinterpret_cast<const float4 *>(p.partial_o + ((size_t)slot * kTileM + r) * D + lane * 4);
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < kBatch; ++q) {
+                const float mnew = fmaxf(mstar[q], fmaxf(ml[0][q].x, ml[1][q].x));
+                if (mnew == -INFINITY) continue;   // nothing seen yet
+                const float keep = mstar[q] == -INFINITY ? 0.f : exp2f(mstar[q] - mnew);
+                lstar[q] *= keep;
+                acc[q].x *= keep; acc[q].y *= keep; acc[q].z *= keep; acc[q].w *= keep;
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const float wgt = ml[k][q].x == -INFINITY ? 0.f : exp2f(ml[k][q].x - mnew);
+                    lstar[q] = fmaf(ml[k][q].y, wgt, lstar[q]);
+                    acc[q].x = fmaf(o[k][q].x, wgt, acc[q].x);
+                    acc[q].y = fmaf(o[k][q].y, wgt, acc[q].y);
+                    acc[q].z = fmaf(o[k][q].z, wgt, acc[q].z);
+                    acc[q].w = fmaf(o[k][q].w, wgt, acc[q].w);
+                }
+                mstar[q] = mnew;
             }
         }
-        const float inv = 1.f / lstar;
-        const int grow = mt * kTileM + r;
-        const int j = grow / p.G, hq = h * p.G + grow % p.G;
-        __nv_bfloat16 *dst = p.out + (((size_t)b * p.T + j) * p.Hq + hq) * D;
-        if (lane * 4 < D) {
-            __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-            __nv_bfloat162 c2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-            uint2 v;
-            v.x = *reinterpret_cast<uint32_t *>(&a);
-            v.y = *reinterpret_cast<uint32_t *>(&c2);
-            *reinterpret_cast<uint2 *>(dst + lane * 4) = v;
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            const int r = r0 + q;
+            if (r >= rows) break;
+            const float inv = 1.f / lstar[q];
+            const int grow = d.mt * kTileM + r;
+            const int j = grow / p.G, hq = d.h * p.G + grow % p.G;
+            __nv_bfloat16 *dst = p.out + (((size_t)d.b * p.T + j) * p.Hq + hq) * D;
+            if (has_cols) {
+                __nv_bfloat162 a = __floats2bfloat162_rn(acc[q].x * inv, acc[q].y * inv);
+                __nv_bfloat162 c2 = __floats2bfloat162_rn(acc[q].z * inv, acc[q].w * inv);
+                uint2 v;
+                v.x = *reinterpret_cast<uint32_t *>(&a);
+                v.y = *reinterpret_cast<uint32_t *>(&c2);
+                *reinterpret_cast<uint2 *>(dst + lane * 4) = v;
+            }
+            if (p.lse && lane == 0)
+                p.lse[((size_t)d.b * p.T + j) * p.Hq + hq] = (mstar[q] + log2f(lstar[q])) * 0.6931471805599453f;
         }
-        if (p.lse && lane == 0)
-            p.lse[((size_t)b * p.T + j) * p.Hq + hq] = (mstar + log2f(lstar)) * 0.6931471805599453f;
     }
 }
 
 void launch_combine(const AttnParams &p, cudaStream_t st) {
-    const int units = p.B * p.sched.units_per_seq;
-    if (units > 0) combine_kernel<<<dim3(units, kTileM / 4), 128, 0, st>>>(p);
+    if (p.B > 0) combine_kernel<<<p.sched.n_ctas, kCombineWarps * 32, 0, st>>>(p);
 }
 
 }  // namespace reader

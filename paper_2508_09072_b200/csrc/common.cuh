@@ -107,6 +107,22 @@ __device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
     return c;
 }
 
+// Written by the attention CTA that starts a unit it does not finish (at most one per CTA); read by
+// the combine kernel.  b < 0: this CTA started no such unit.
+struct SplitDesc {
+    int32_t b, h, mt, c_last;   // unit, and the last CTA holding one of its partials
+};
+
+// Called by one thread per segment: if the segment starts its unit without finishing it, note where
+// the unit's partials end so that the combine kernel can find them without any search.
+__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, const Segment &g, int cta, int w_seg_begin, int W) {
+    if (g.tile_begin != 0 || g.full) return;
+    SplitDesc d;
+    d.b = g.b; d.h = g.h; d.mt = g.mt;
+    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, s.n_ctas, W);
+    desc[cta] = d;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Attention parameters
 // ---------------------------------------------------------------------------------------------
@@ -119,6 +135,7 @@ struct AttnParams {
     float *lse;                // nullable
     float *partial_o;          // [slots][kTileM][D]
     float *partial_ml;         // [slots][kTileM][2]  (m in log2 units, l)
+    SplitDesc *split_desc;     // [n_ctas]
     int32_t *status;           // [B]
     int32_t *error_flag;       // one word in the workspace: set on a bounded-wait timeout
     int B, T, Hq, Hkv, D, G;
@@ -136,7 +153,7 @@ void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int3
 void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
                     int units_per_seq, uint64_t *anc_out /*nullable*/, int32_t *seq_tile_start,
                     int32_t *seq_ntiles, int32_t *seq_npages, int32_t *status, int32_t *error_flag,
-                    cudaStream_t st);
+                    __nv_bfloat16 *out, float *lse /*nullable*/, int Hq, int D, cudaStream_t st);
 void launch_attn_generic(const AttnParams &p, cudaStream_t st);
 void launch_combine(const AttnParams &p, cudaStream_t st);
 void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits, float *part_val,

@@ -45,7 +45,9 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
                                                        int32_t *__restrict__ seq_ntiles,
                                                        int32_t *__restrict__ seq_npages,
                                                        int32_t *__restrict__ status,
-                                                       int32_t *__restrict__ error_flag) {
+                                                       int32_t *__restrict__ error_flag,
+                                                       __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
+                                                       int Hq, int D) {
     __shared__ int32_t par[32][kMaxNodes];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) *error_flag = 0;
@@ -82,6 +84,13 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
             seq_ntiles[b] = st == READER_OK ? npages + n_tree_tiles : 0;
             seq_npages[b] = st == READER_OK ? npages : 0;
         }
+        if (st != READER_OK) {   // a rejected sequence gets defined output: zero rows, zero lse
+            const size_t n16 = (size_t)T * Hq * D / 8;
+            uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)b * T * Hq * D);
+            for (size_t i = lane; i < n16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+            if (lse)
+                for (int i = lane; i < T * Hq; i += 32) lse[(size_t)b * T * Hq + i] = 0.f;
+        }
         __syncwarp();
     }
     __syncthreads();
@@ -104,10 +113,11 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
 
 void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
                     int units_per_seq, uint64_t *anc_out, int32_t *seq_tile_start, int32_t *seq_ntiles,
-                    int32_t *seq_npages, int32_t *status, int32_t *error_flag, cudaStream_t st) {
+                    int32_t *seq_npages, int32_t *status, int32_t *error_flag, __nv_bfloat16 *out, float *lse,
+                    int Hq, int D, cudaStream_t st) {
     prepare_kernel<<<1, 1024, 0, st>>>(c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages, parent, B, T,
                                        n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles,
-                                       seq_npages, status, error_flag);
+                                       seq_npages, status, error_flag, out, lse, Hq, D);
 }
 
 }  // namespace reader

@@ -379,8 +379,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         int it = 0;
         int w = w_begin;
+        if (tid == 0) p.split_desc[cta].b = -1;
         while (w < w_end) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            if (tid == 0) record_split(p.split_desc, p.sched, sg, cta, w, W);
             w += sg.tile_end - sg.tile_begin;
             const int L = p.seq_lens[sg.b];
             const int grow = sg.mt * kTileM + tid;
@@ -527,6 +529,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                         *reinterpret_cast<uint4 *>(po + c + 4 * i) = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
                 *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)sg.slot * kTileM + tid) * 2) = make_float2(m_used, l);
+
             }
             tc_fence_before();
         }
