@@ -424,13 +424,19 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                         if (!((hi >> i) & 1u)) s1[i] = 0xff800000u;
                     }
                 }
-                float mxs[8];
+                float mxs[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i]));
+                for (int i = 0; i < 4; ++i) mxs[i] = max3(__uint_as_float(s0[i]), __uint_as_float(s1[i]), __uint_as_float(s0[i + 4]));
 #pragma unroll
-                for (int i = 8; i < 32; ++i) mxs[i & 7] = fmaxf(mxs[i & 7], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
-                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
-                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                for (int i = 0; i < 4; ++i) mxs[i] = max3(mxs[i], __uint_as_float(s1[i + 4]), __uint_as_float(s0[i + 8]));
+#pragma unroll
+                for (int i = 8; i < 32; i += 8)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        mxs[q] = max3(mxs[q], __uint_as_float(s1[i + q]), __uint_as_float(s0[i + q + 4]));
+                        mxs[q] = max3(mxs[q], __uint_as_float(s1[i + q + 4]), i + 8 < 32 ? __uint_as_float(s0[i + q + 8]) : -INFINITY);
+                    }
+                const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
                 const float m_new = fmaxf(m_used, mx * p.scale_log2);
                 const bool first = t == sg.tile_begin;
                 const bool raise = __any_sync(0xffffffffu, m_new > m_used + kRaiseMaxBy);
