@@ -11,9 +11,10 @@
 //               run far ahead.  Bytes beyond a sequence's length or the tree's end can never
 //               reach a product: scores there are replaced by -inf, and the value product skips
 //               16-key slices past the end and zeroes the tail of the last slice in place.
-//   warp 5      MMA issuer, event driven: it issues S[i] = Q K[i]^T whenever K[i] has landed and
-//               a score buffer is free, and O += P[j] V[j] whenever P[j] and V[j] are ready; it
-//               never sits on one barrier while the other kind of work could be issued.
+//   warp 5      issues S[i] = Q K[i]^T as soon as K[i] has landed and score buffer i & 1 is free
+//   warp 6      issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Two issuing warps because
+//               one thread can start a tcgen05.mma only every ~120 cycles: with 8 + 4 of them per
+//               tile a single issuer was the bottleneck of the whole kernel.
 //   warps 0-3   softmax: thread r owns query row r = TMEM lane r.  Scores come from TMEM, the
 //               ancestor bitmask / length mask is applied, the running maximum is raised only
 //               when it grows by more than 2^8 (the accumulator in TMEM is rescaled then),
@@ -38,9 +39,10 @@ namespace {
 using namespace ptx;
 
 constexpr int kStages = 2;          // per CTA; two CTAs share an SM, so four tiles are in flight per SM
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kProducerWarp = 4;
-constexpr int kMmaWarp = 5;
+constexpr int kMmaWarp = 5;   // issues the score products, owns the TMEM allocation
+constexpr int kPvWarp = 6;    // issues the value products
 constexpr uint64_t kWaitLimitNs = 1000000000ull;
 constexpr float kRaiseMaxBy = 8.f;   // log2 units
 constexpr uint32_t kTmemCols = 256;
@@ -64,7 +66,7 @@ struct Cfg {
 
 struct Bars {
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full, pv_done;
+    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full[2], pv_done;
     uint32_t tmem_base;
     int32_t abort;
 };
@@ -205,9 +207,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         mbar_init(bar(&bars->q_empty), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(&bars->s_full[s]), 1);
-            mbar_init(bar(&bars->s_empty[s]), kTileM);
+            mbar_init(bar(&bars->s_empty[s]), 1);
         }
-        mbar_init(bar(&bars->p_full), kTileM);
+        mbar_init(bar(&bars->p_full[0]), kTileM);
+        mbar_init(bar(&bars->p_full[1]), kTileM);
         mbar_init(bar(&bars->pv_done), 1);
         bars->abort = 0;
         fence_mbar_init();
@@ -291,88 +294,87 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 }
         }
     } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ score-product issuer
+        // (one thread can start a tcgen05.mma only every ~120 cycles, so the two kinds of product
+        // are issued by two warps)
         constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kPage, false, false);
-        constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, false, true);
         // descriptors differ only in their start-address field (bytes >> 4), so each operand's
         // descriptor is one addition away from a base built once
         const uint64_t descQ = smem_desc_sw128(sQ, 16, 1024), descK = smem_desc_sw128(sK, 16, 1024);
-        const uint64_t descP = smem_desc_sw128(sP, 16, 1024), descV = smem_desc_sw128(sV, C::kHalfRowsKV, 1024);
-        int it0 = 0, seg = 0;
+        int i = 0, seg = 0;
         int w = w_begin;
-        Watchdog dog;
+        while (w < w_end && !*abort_s) {
+            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            const int n = sg.tile_end - sg.tile_begin;
+            w += n;
+            wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
+            for (int t = 0; t < n; ++t, ++i) {
+                const int stage = i % kStages, buf = i & 1;
+                wait(bar(&bars->k_full[stage]), (i / kStages) & 1, abort_s, p.error_flag);
+                // score buffer i & 1 holds P[i-2] until that value product has read it
+                wait(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1, abort_s, p.error_flag);
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint64_t kd = descK + (uint64_t)((stage * C::kTileBytes) >> 4);
+#pragma unroll
+                    for (int hf = 0; hf < C::kHalves; ++hf)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_bf16_ss(tmem + buf * kPage, descQ + (uint64_t)((hf * C::kHalfRowsQ + kk * 32) >> 4),
+                                        kd + (uint64_t)((hf * C::kHalfRowsKV + kk * 32) >> 4), kIdescQK, (hf | kk) != 0);
+                    mma_commit(bar(&bars->k_empty[stage]));
+                    mma_commit(bar(&bars->s_full[buf]));
+                    if (t == n - 1) mma_commit(bar(&bars->q_empty));
+                }
+                __syncwarp();
+            }
+            ++seg;
+        }
+    } else if (warp == kPvWarp) {
+        // ------------------------------------------------------------------ value-product issuer
+        constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, false, true);
+        const uint64_t descV = smem_desc_sw128(sV, C::kHalfRowsKV, 1024);
+        int i = 0;
+        int w = w_begin;
         while (w < w_end && !*abort_s) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += n;
             const int L = p.seq_lens[sg.b];
-            wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
-            tc_fence_after();
-            int next_qk = 0, next_pv = 0;
-            while (next_pv < n) {
-                bool moved = false;
-                if (next_qk < n) {
-                    const int i = it0 + next_qk, stage = i % kStages, buf = i & 1;
-                    if (ready(bar(&bars->k_full[stage]), (i / kStages) & 1) &&
-                        ready(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1)) {
-                        tc_fence_after();
-                        if (lane == 0) {
-                            const uint64_t kd = descK + (uint64_t)((stage * C::kTileBytes) >> 4);
-#pragma unroll
-                            for (int hf = 0; hf < C::kHalves; ++hf)
-#pragma unroll
-                                for (int kk = 0; kk < 4; ++kk)
-                                    mma_bf16_ss(tmem + buf * kPage, descQ + (uint64_t)((hf * C::kHalfRowsQ + kk * 32) >> 4),
-                                                kd + (uint64_t)((hf * C::kHalfRowsKV + kk * 32) >> 4), kIdescQK, (hf | kk) != 0);
-                            mma_commit(bar(&bars->k_empty[stage]));
-                            mma_commit(bar(&bars->s_full[buf]));
-                            if (next_qk == n - 1) mma_commit(bar(&bars->q_empty));
-                        }
-                        __syncwarp();
-                        ++next_qk;
-                        moved = true;
+            for (int tl = 0; tl < n; ++tl, ++i) {
+                const int stage = i % kStages;
+                wait(bar(&bars->p_full[i & 1]), (i >> 1) & 1, abort_s, p.error_flag);
+                wait(bar(&bars->v_full[stage]), (i / kStages) & 1, abort_s, p.error_flag);
+                tc_fence_after();
+                const uint32_t vbase = sV + stage * C::kTileBytes;
+                // keys past the end of the sequence / tree: whole 16-key slices are not multiplied at
+                // all, the rest of the last slice is zeroed in place
+                const int t = sg.tile_begin + tl;
+                const int valid = t < sg.npages ? min(kPage, L - t * kPage) : min(kPage, p.T - (t - sg.npages) * kPage);
+                const int slices = (valid + 15) >> 4;
+                if (valid & 15) {
+                    constexpr int kChunks = D / 8;
+                    for (int idx = lane; idx < (slices * 16 - valid) * kChunks; idx += 32) {
+                        const int rr = valid + idx / kChunks, cc = idx % kChunks;
+                        const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
                     }
+                    fence_proxy_async();
+                    __syncwarp();
                 }
-                if (next_pv < next_qk) {
-                    const int i = it0 + next_pv, stage = i % kStages;
-                    if (ready(bar(&bars->p_full), i & 1) && ready(bar(&bars->v_full[stage]), (i / kStages) & 1)) {
-                        tc_fence_after();
-                        const uint32_t vbase = sV + stage * C::kTileBytes;
-                        // keys past the end of the sequence / tree: whole 16-key slices are not
-                        // multiplied at all, the rest of the last slice is zeroed in place
-                        const int t = sg.tile_begin + next_pv;
-                        const int valid = t < sg.npages ? min(kPage, L - t * kPage) : min(kPage, p.T - (t - sg.npages) * kPage);
-                        const int slices = (valid + 15) >> 4;
-                        if (valid & 15) {
-                            constexpr int kChunks = D / 8;
-                            for (int idx = lane; idx < (slices * 16 - valid) * kChunks; idx += 32) {
-                                const int rr = valid + idx / kChunks, cc = idx % kChunks;
-                                const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
-                            }
-                            fence_proxy_async();
-                            __syncwarp();
-                        }
-                        if (lane == 0) {
-                            const uint64_t vd = descV + (uint64_t)((stage * C::kTileBytes) >> 4);
+                if (lane == 0) {
+                    const uint64_t vd = descV + (uint64_t)((stage * C::kTileBytes) >> 4);
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                if (kk < slices)
-                                    mma_bf16_ss(tmem + kTmemO, descP + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4),
-                                                kIdescPV, (next_pv | kk) != 0);
-                            mma_commit(bar(&bars->v_empty[stage]));
-                            mma_commit(bar(&bars->pv_done));
-                        }
-                        __syncwarp();
-                        ++next_pv;
-                        moved = true;
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        if (kk < slices)
+                            mma_bf16_ts(tmem + kTmemO, tmem + (i & 1) * kPage + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                                        kIdescPV, (tl | kk) != 0);
+                    mma_commit(bar(&bars->v_empty[stage]));
+                    mma_commit(bar(&bars->s_empty[i & 1]));
+                    mma_commit(bar(&bars->pv_done));
                 }
-                if (moved) dog.progress();
-                else if (dog.expired(abort_s, p.error_flag)) break;
+                __syncwarp();
             }
-            it0 += n;
-            ++seg;
         }
     } else {
         // ------------------------------------------------------------------ softmax / epilogue
@@ -413,8 +415,6 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 tmem_ld32(tmem + lane_base + buf * kPage, s0);
                 tmem_ld32(tmem + lane_base + buf * kPage + 32, s1);
                 tmem_wait_ld();
-                tc_fence_before();
-                mbar_arrive(bar(&bars->s_empty[buf]));
 
                 if (vis != ~0ull) {
                     const uint32_t lo = (uint32_t)vis, hi = (uint32_t)(vis >> 32);
@@ -467,12 +467,11 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 }
                 l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
 
-                // the previous value product must be complete before P or O are touched
-                if (it > 0) {
+                if (raise && !first) {
+                    // O may only be rescaled once the previous value product is complete (the scores of
+                    // this tile exist, so product it-2 is complete and the parity wait is unambiguous)
                     wait(bar(&bars->pv_done), (it - 1) & 1, abort_s, p.error_flag);
                     tc_fence_after();
-                }
-                if (raise && !first) {
 #pragma unroll 1
                     for (int c = 0; c < D; c += 32) {
                         uint32_t o[32];
@@ -484,17 +483,20 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                     }
                     tmem_wait_st();
                 }
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t off = tid * 128 + ((c ^ (tid & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + off), "r"(pk[4 * c]), "r"(pk[4 * c + 1]), "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
-                }
-                fence_proxy_async();
+                // P (bf16 pairs) replaces the scores it was computed from: 32 columns of this buffer
+                tmem_st32(tmem + lane_base + buf * kPage, pk);
+                tmem_wait_st();
+                // one barrier per score buffer: a warp may be a tile ahead of a slower one (never two,
+                // the next scores for this buffer wait for this tile's value product)
                 tc_fence_before();
-                mbar_arrive(bar(&bars->p_full));
+                mbar_arrive(bar(&bars->p_full[buf]));
             }
 
             // ---- segment epilogue
+            // A parity wait can only tell the barrier's current phase from the one before it.  This
+            // warp may have run a tile ahead, so all it knows is that product it-3 is complete: it
+            // waits for product it-2 first, then for the last one.
+            if (it >= 2) wait(bar(&bars->pv_done), (it - 2) & 1, abort_s, p.error_flag);
             wait(bar(&bars->pv_done), (it - 1) & 1, abort_s, p.error_flag);
             tc_fence_after();
             if (sg.full) {
