@@ -37,7 +37,8 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
     if (d.b < 0) return;
     const int rows = min(kTileM, p.T * p.G - d.mt * kTileM);
     const bool has_cols = lane * 4 < D;
-    const bool all_live = W >= p.sched.n_ctas;   // with fewer tiles than CTAs some ranges are empty
+    const int n_ctas = effective_ctas(p.sched.n_ctas, W);
+    const bool all_live = W >= n_ctas;   // with fewer tiles than CTAs some ranges are empty
 
     for (int rb = 0; rb < kRowsPerWarp; rb += kBatch) {
         const int r0 = warp * kRowsPerWarp + rb;
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
             for (int k = 0; k < 2; ++k) {
                 const int c = cb + k;
                 // a CTA with an empty range wrote nothing
-                const bool live = c <= d.c_last && (all_live || range_begin(c + 1, p.sched.n_ctas, W) != range_begin(c, p.sched.n_ctas, W));
+                const bool live = c <= d.c_last && (all_live || range_begin(c + 1, n_ctas, W) != range_begin(c, n_ctas, W));
                 const int slot = c == c0 ? 2 * c + 1 : 2 * c;
 #pragma unroll
                 for (int q = 0; q < kBatch; ++q) {

@@ -28,7 +28,7 @@ struct Sched {
     const int32_t *seq_tile_start;  // [B+1] first flat tile of sequence b
     const int32_t *seq_ntiles;      // [B]   tiles per unit of sequence b (0: sequence skipped)
     const int32_t *seq_npages;      // [B]   committed pages among them
-    int32_t n_ctas;
+    int32_t n_ctas;                 // CTAs launched; effective_ctas() of them share the work
     int32_t units_per_seq;          // Hkv * n_mtiles
     int32_t n_mtiles;
 };
@@ -41,8 +41,18 @@ struct Segment {
     int slot;                  // partial slot when !full
 };
 
+constexpr int kMinTilesPerCta = 8;
+
+// CTAs that share the W tiles of a call: all that were launched, unless that would leave fewer than
+// kMinTilesPerCta tiles each (start-up, epilogue and the merge of partials cost several tiles' time,
+// so a small call is better cut into few pieces).  The rest find an empty range.
+__device__ __forceinline__ int effective_ctas(int n_launched, int W) {
+    return max(1, min(n_launched, (W + kMinTilesPerCta - 1) / kMinTilesPerCta));
+}
+
+// First tile of CTA c's range; c >= n_ctas (a CTA left without work) gets W.
 __device__ __forceinline__ int range_begin(int c, int n_ctas, int W) {
-    return (int)(((int64_t)c * W) / n_ctas);
+    return c >= n_ctas ? W : (int)(((int64_t)c * W) / n_ctas);
 }
 
 // Largest b with seq_tile_start[b] <= w (w < W).
@@ -115,11 +125,11 @@ struct SplitDesc {
 
 // Called by one thread per segment: if the segment starts its unit without finishing it, note where
 // the unit's partials end so that the combine kernel can find them without any search.
-__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, const Segment &g, int cta, int w_seg_begin, int W) {
+__device__ __forceinline__ void record_split(SplitDesc *desc, int n_ctas, const Segment &g, int cta, int w_seg_begin, int W) {
     if (g.tile_begin != 0 || g.full) return;
     SplitDesc d;
     d.b = g.b; d.h = g.h; d.mt = g.mt;
-    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, s.n_ctas, W);
+    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, n_ctas, W);
     desc[cta] = d;
 }
 
