@@ -4,8 +4,7 @@
 // unit (sequence, KV head, 128 query rows) a CTA computes S = Q K^T and O += P V with tcgen05.mma,
 // one KV tile of 64 keys (one cache page, or 64 tree nodes) at a time:
 //
-//   warp 4      producer: K tiles and V tiles travel through two separate rings of kStages
-//               slots.  Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages
+//   warp 4      producer: K tiles and V tiles travel through two separate rings (3 and 2 slots).  Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages
 //               from the pool, tree tiles from the tree tensors.  A K slot is free again as soon
 //               as its score product has run, long before the tile's value product, so key loads
 //               run far ahead.  Bytes beyond a sequence's length or the tree's end can never
@@ -18,13 +17,15 @@
 //   warps 0-3   softmax: thread r owns query row r = TMEM lane r.  Scores come from TMEM, the
 //               ancestor bitmask / length mask is applied, the running maximum is raised only
 //               when it grows by more than 2^8 (the accumulator in TMEM is rescaled then),
-//               probabilities go to shared memory as the bf16 A operand of the value product.
+//               probabilities (bf16 pairs) are written over the scores they came from and are
+//               the value product's A operand straight from tensor memory.
 //               The same threads write O (or an (m, l, O) partial) at the end of a segment.
 // The 128 query rows of a unit (node j, group member g -> row j*G+g) come in by one 4-D TMA box per
 // 64 columns, issued by the producer as soon as the previous segment's last score product is done.
 //
-// TMEM: columns 0-127 hold two score buffers of 64 columns, columns 128.. hold O (head_dim
-// columns), all fp32, lane = query row.  Every wait on an mbarrier is bounded: after one second
+// TMEM: columns 0-127 hold two score buffers of 64 columns (fp32; the first 32 columns of a buffer
+// hold P as bf16 pairs once its softmax is done), columns 128.. hold O (head_dim columns, fp32);
+// lane = query row.  Every wait on an mbarrier is bounded: after one second
 // without progress a CTA raises the error flag in the workspace, stops waiting and runs to its end.
 #include <cuda.h>
 
@@ -38,7 +39,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kStages = 2;          // per CTA; two CTAs share an SM, so four tiles are in flight per SM
+constexpr int kStagesK = 3;         // K tiles in flight per CTA (two CTAs share an SM)
+constexpr int kStagesV = 2;         // V tiles
 constexpr int kThreads = 224;
 constexpr int kProducerWarp = 4;
 constexpr int kMmaWarp = 5;   // issues the score products, owns the TMEM allocation
@@ -54,18 +56,16 @@ struct Cfg {
     static constexpr int kHalfRowsQ = kTileM * 128;        // bytes of one 64-column block of Q
     static constexpr int kHalfRowsKV = kPage * 128;        // bytes of one 64-column block of a KV tile
     static constexpr int kQBytes = kTileM * D * 2;
-    static constexpr int kPBytes = kTileM * kPage * 2;
     static constexpr int kTileBytes = kPage * D * 2;
     static constexpr int kOffQ = 0;
-    static constexpr int kOffP = kQBytes;
-    static constexpr int kOffK = kOffP + kPBytes;                 // ring of K tiles
-    static constexpr int kOffV = kOffK + kStages * kTileBytes;    // ring of V tiles
-    static constexpr int kOffBars = kOffV + kStages * kTileBytes;
+    static constexpr int kOffK = kQBytes;                          // ring of K tiles
+    static constexpr int kOffV = kOffK + kStagesK * kTileBytes;    // ring of V tiles
+    static constexpr int kOffBars = kOffV + kStagesV * kTileBytes;
     static constexpr int kSmemBytes = kOffBars + 256;   // + barriers; two CTAs of head_dim 128 fit one SM
 };
 
 struct Bars {
-    uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+    uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
     uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full[2], pv_done;
     uint32_t tmem_base;
     int32_t abort;
@@ -193,13 +193,15 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
 
-    const uint32_t sQ = base + C::kOffQ, sP = base + C::kOffP, sK = base + C::kOffK, sV = base + C::kOffV;
+    const uint32_t sQ = base + C::kOffQ, sK = base + C::kOffK, sV = base + C::kOffV;
     auto bar = [&](const uint64_t *b) { return smem_u32(b); };
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStagesK; ++s) {
             mbar_init(bar(&bars->k_full[s]), 1);
             mbar_init(bar(&bars->k_empty[s]), 1);
+        }
+        for (int s = 0; s < kStagesV; ++s) {
             mbar_init(bar(&bars->v_full[s]), 1);
             mbar_init(bar(&bars->v_empty[s]), 1);
         }
@@ -264,8 +266,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 moved = true;
             }
             if (kc.active) {
-                const int stage = kc.it % kStages;
-                if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStages) & 1) ^ 1)) {
+                const int stage = kc.it % kStagesK;
+                if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStagesK) & 1) ^ 1)) {
                     load_tile<D>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane);
                     __syncwarp();
                     kc.advance(p, cta, lane);
@@ -273,8 +275,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 }
             }
             if (vc.active) {
-                const int stage = vc.it % kStages;
-                if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStages) & 1) ^ 1)) {
+                const int stage = vc.it % kStagesV;
+                if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStagesV) & 1) ^ 1)) {
                     load_tile<D>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane);
                     __syncwarp();
                     vc.advance(p, cta, lane);
@@ -287,11 +289,11 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         // a CTA that gave up must not exit under its own copies: let the last ones land (bounded)
         if (*abort_s) {
             const uint64_t t0 = globaltimer_ns();
-            for (int i = max(0, kc.it - kStages); i < kc.it; ++i)
-                while (!mbar_try_wait(bar(&bars->k_full[i % kStages]), (i / kStages) & 1) && globaltimer_ns() - t0 < 20000000ull) {
+            for (int i = max(0, kc.it - kStagesK); i < kc.it; ++i)
+                while (!mbar_try_wait(bar(&bars->k_full[i % kStagesK]), (i / kStagesK) & 1) && globaltimer_ns() - t0 < 20000000ull) {
                 }
-            for (int i = max(0, vc.it - kStages); i < vc.it; ++i)
-                while (!mbar_try_wait(bar(&bars->v_full[i % kStages]), (i / kStages) & 1) && globaltimer_ns() - t0 < 20000000ull) {
+            for (int i = max(0, vc.it - kStagesV); i < vc.it; ++i)
+                while (!mbar_try_wait(bar(&bars->v_full[i % kStagesV]), (i / kStagesV) & 1) && globaltimer_ns() - t0 < 20000000ull) {
                 }
         }
     } else if (warp == kMmaWarp) {
@@ -310,8 +312,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             w += n;
             wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
             for (int t = 0; t < n; ++t, ++i) {
-                const int stage = i % kStages, buf = i & 1;
-                wait(bar(&bars->k_full[stage]), (i / kStages) & 1, abort_s, p.error_flag);
+                const int stage = i % kStagesK, buf = i & 1;
+                wait(bar(&bars->k_full[stage]), (i / kStagesK) & 1, abort_s, p.error_flag);
                 // score buffer i & 1 holds P[i-2] until that value product has read it
                 wait(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1, abort_s, p.error_flag);
                 tc_fence_after();
@@ -343,9 +345,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             w += n;
             const int L = p.seq_lens[sg.b];
             for (int tl = 0; tl < n; ++tl, ++i) {
-                const int stage = i % kStages;
+                const int stage = i % kStagesV;
                 wait(bar(&bars->p_full[i & 1]), (i >> 1) & 1, abort_s, p.error_flag);
-                wait(bar(&bars->v_full[stage]), (i / kStages) & 1, abort_s, p.error_flag);
+                wait(bar(&bars->v_full[stage]), (i / kStagesV) & 1, abort_s, p.error_flag);
                 tc_fence_after();
                 const uint32_t vbase = sV + stage * C::kTileBytes;
                 // keys past the end of the sequence / tree: whole 16-key slices are not multiplied at
