@@ -183,6 +183,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = G;
     p.max_pages = cache->max_pages_per_seq;
     p.num_pages = cache->num_pages;
+    p.shared_prefix_pages = cache->shared_prefix_len / kPage;
     p.scale_log2 = softmax_scale * 1.4426950408889634f;
     p.sched.seq_tile_start = reinterpret_cast<const int32_t *>(ws + w.seq_tile_start);
     p.sched.seq_ntiles = reinterpret_cast<const int32_t *>(ws + w.seq_ntiles);

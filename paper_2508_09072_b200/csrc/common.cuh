@@ -150,6 +150,7 @@ struct AttnParams {
     int32_t *error_flag;       // one word in the workspace: set on a bounded-wait timeout
     int B, T, Hq, Hkv, D, G;
     int max_pages, num_pages;
+    int shared_prefix_pages;   // leading page-table entries common to every sequence
     float scale_log2;          // softmax_scale * log2(e)
     Sched sched;
 };

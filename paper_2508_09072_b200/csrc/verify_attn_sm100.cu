@@ -159,7 +159,8 @@ struct TileCursor {
 // side never multiplies them (see the MMA issuer).  Called by the whole producer warp.
 template <int D>
 __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor &c, const CUtensorMap *pool_map,
-                                          const CUtensorMap *tree_map, uint32_t dst, uint32_t full, int lane) {
+                                          const CUtensorMap *tree_map, uint32_t dst, uint32_t full, int lane,
+                                          uint64_t stream_policy, int first_streamed_tile) {
     using C = Cfg<D>;
     const int page = c.page();
     if (lane != 0) return;
@@ -167,7 +168,11 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor 
     if (c.t < c.sg.npages) {
         const int row = (page * p.Hkv + c.sg.h) * kPage;
 #pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf) tma_load_2d(dst + hf * C::kHalfRowsKV, pool_map, full, hf * 64, row);
+        for (int hf = 0; hf < C::kHalves; ++hf) {
+            // a page that no other CTA will read again should not push reusable lines out of L2
+            if (c.t >= first_streamed_tile) tma_load_2d_hint(dst + hf * C::kHalfRowsKV, pool_map, full, hf * 64, row, stream_policy);
+            else tma_load_2d(dst + hf * C::kHalfRowsKV, pool_map, full, hf * 64, row);
+        }
     } else {
         const int node0 = c.sg.b * p.T + (c.t - c.sg.npages) * kPage;
 #pragma unroll
@@ -241,6 +246,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             prefetch_tensormap(&vtmap);
             prefetch_tensormap(&qmap);
         }
+        // pages are read exactly once when a KV head has a single M tile and nothing is shared (with a
+        // shared prefix the hint measured slightly slower, so it is left off there)
+        const uint64_t stream_policy = l2_policy_evict_first();
+        const int first_streamed_tile = (p.sched.n_mtiles == 1 && p.shared_prefix_pages == 0) ? 0 : 0x7fffffff;
         TileCursor kc, vc;
         kc.init(p, cta, lane, w_begin, w_end);
         vc.init(p, cta, lane, w_begin, w_end);
@@ -268,7 +277,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (kc.active) {
                 const int stage = kc.it % kStagesK;
                 if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStagesK) & 1) ^ 1)) {
-                    load_tile<D>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane);
+                    load_tile<D>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     kc.advance(p, cta, lane);
                     moved = true;
@@ -277,7 +286,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (vc.active) {
                 const int stage = vc.it % kStagesV;
                 if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStagesV) & 1) ^ 1)) {
-                    load_tile<D>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane);
+                    load_tile<D>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     vc.advance(p, cta, lane);
                     moved = true;
