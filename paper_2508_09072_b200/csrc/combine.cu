@@ -17,6 +17,7 @@ constexpr int kRowsPerWarp = kTileM / kCombineWarps;    // 8 rows, merged in bat
 constexpr int kBatch = 2;
 
 __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const AttnParams p) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // launched ahead of the attention kernel's end
     const int c0 = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.D;
@@ -113,7 +114,17 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
 }
 
 void launch_combine(const AttnParams &p, cudaStream_t st) {
-    if (p.B > 0) combine_kernel<<<p.sched.n_ctas, kCombineWarps * 32, 0, st>>>(p);
+    if (p.B <= 0) return;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.sched.n_ctas);
+    cfg.blockDim = dim3(kCombineWarps * 32);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, combine_kernel, p);
 }
 
 }  // namespace reader

@@ -191,6 +191,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// Programmatic dependent launch: wait until the grids this one depends on have completed and their
+// writes are visible (no-op for a kernel launched the ordinary way) / let dependents start launching.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

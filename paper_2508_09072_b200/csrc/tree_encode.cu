@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
                                                        int Hq, int D) {
     __shared__ int32_t par[32][kMaxNodes];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may set itself up meanwhile
     if (threadIdx.x == 0) *error_flag = 0;
     for (int b = warp; b < B; b += 32) {
         for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];

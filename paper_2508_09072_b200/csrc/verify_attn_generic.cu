@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(kTileM) attn_generic_kernel(const AttnParams p
     constexpr int kChunks = D / 8;                                      // 16-byte chunks per row
 
     const int cta = blockIdx.x, tid = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int W = p.sched.seq_tile_start[p.B];
     const int n_ctas = effective_ctas(p.sched.n_ctas, W);
     const int w_end = range_begin(cta + 1, n_ctas, W);

@@ -232,6 +232,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
+    // everything above overlapped the preparation kernel; its results are read from here on
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int W = p.sched.seq_tile_start[p.B];
     const int n_ctas = effective_ctas(p.sched.n_ctas, W);
     const int w_begin = range_begin(cta, n_ctas, W);
@@ -690,10 +693,23 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_
         }
         m->q = p.q; m->qB = p.B; m->qT = p.T; m->qHq = p.Hq; m->qG = p.G; m->qD = p.D;
     }
-    if (p.D == 128)
-        attn_sm100_kernel<128><<<p.sched.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
-    else
-        attn_sm100_kernel<64><<<p.sched.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.sched.n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = p.D == 128 ? Cfg<128>::kSmemBytes : Cfg<64>::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // prologue overlaps the preparation kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = p.D == 128
+        ? cudaLaunchKernelEx(&cfg, attn_sm100_kernel<128>, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap)
+        : cudaLaunchKernelEx(&cfg, attn_sm100_kernel<64>, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return READER_ERR_CUDA;
+    }
     return READER_OK;
 }
 
