@@ -231,14 +231,10 @@ def run_ours(args):
     def mk():
         return torch.cuda.Event(enable_timing=True)
 
-    # ---- device-resident timing
+    # ---- device-resident timing: K steps back to back, nothing but the library's launches in between
     for _ in range(max(args.warmup, 3)):
         step()
     K = args.steps
-    evs = [[mk() for _ in range(4)] for _ in range(K)]
-    kev = [(mk(), mk()) for _ in range(K)]
-    for a, b in kev:                                  # create the handles
-        a.record(); b.record()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -247,19 +243,31 @@ def run_ours(args):
     e0, e1 = mk(), mk()
     e0.record()
     for i in range(K):
-        rd.set_timing_events(*kev[i])
-        step(evs[i])
+        step()
     e1.record()
     barrier()
     t_wall1 = time.time()
-    rd.set_timing_events(None, None)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
-    t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / K
-    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / K
-    t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / K
-    t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / K
     assert int(status.max().item()) == 0 and int(cstat.max().item()) == 0 and int(acc_out[3].max().item()) == 0
+
+    # ---- per-call and per-kernel breakdown: a second, shorter loop with events between the calls and,
+    # inside reader_verify_attn, around the attention kernel (events between two kernels switch the
+    # overlap of their launches off, so this loop is a little slower than the one above)
+    Kb = max(3, min(K, 300))
+    evs = [[mk() for _ in range(4)] for _ in range(Kb)]
+    kev = [(mk(), mk()) for _ in range(Kb)]
+    for a, b in kev:                                  # create the handles
+        a.record(); b.record()
+    for i in range(Kb):
+        rd.set_timing_events(*kev[i])
+        step(evs[i])
+    barrier()
+    rd.set_timing_events(None, None)
+    t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / Kb
+    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / Kb
+    t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / Kb
+    t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
 
     # ---- end to end: host buffers in, results out, every step
     host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits")}
