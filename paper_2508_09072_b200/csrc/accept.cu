@@ -24,6 +24,8 @@ template <bool kVec>
 __global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ logits, int64_t vocab, int chunk,
                                                      int splits, float *__restrict__ part_val,
                                                      int32_t *__restrict__ part_idx) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int64_t row = blockIdx.x;
     const int split = blockIdx.y;
     const int c0 = split * chunk;
@@ -86,9 +88,9 @@ void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits,
     chunk = (chunk + 3) & ~3;
     dim3 grid((unsigned)rows, (unsigned)splits);
     if (vocab % 4 == 0)
-        argmax_kernel<true><<<grid, 256, 0, st>>>(logits, vocab, chunk, splits, part_val, part_idx);
+        launch_pdl(argmax_kernel<true>, grid, dim3(256), 0, st, logits, vocab, chunk, splits, part_val, part_idx);
     else
-        argmax_kernel<false><<<grid, 256, 0, st>>>(logits, vocab, chunk, splits, part_val, part_idx);
+        launch_pdl(argmax_kernel<false>, grid, dim3(256), 0, st, logits, vocab, chunk, splits, part_val, part_idx);
 }
 
 // One warp per sequence.
@@ -100,6 +102,8 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t *__restrict__
                                                      int32_t *__restrict__ bonus, int32_t *__restrict__ status) {
     __shared__ int32_t par_s[4][kMaxNodes];
     __shared__ int32_t tgt_s[4][kMaxNodes];
+    pdl_wait();
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * 4 + warp;
     if (b >= B) return;
@@ -175,7 +179,7 @@ void launch_accept(const int32_t *parent, const int32_t *tok, int32_t *target, i
                    const float *part_val, const int32_t *part_idx, int splits, int32_t *path, int32_t *n_acc,
                    int32_t *bonus, int32_t *status, cudaStream_t st) {
     if (B <= 0) return;
-    accept_kernel<<<(B + 3) / 4, 128, 0, st>>>(parent, tok, target, B, T, max_path, part_val, part_idx, splits,
+    launch_pdl(accept_kernel, dim3((B + 3) / 4), dim3(128), 0, st, parent, tok, target, B, T, max_path, part_val, part_idx, splits,
                                                path, n_acc, bonus, status);
 }
 

@@ -17,6 +17,8 @@ __global__ void __launch_bounds__(256) kv_commit_kernel(__nv_bfloat16 *__restric
                                                         const int32_t *__restrict__ n_acc, int max_path,
                                                         int update_seq_lens, int32_t *__restrict__ slots,
                                                         int32_t *__restrict__ status) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int b = blockIdx.x, tid = threadIdx.x;
     __shared__ int ok_s;
     const int L = seq_lens[b];
@@ -69,7 +71,7 @@ void launch_kv_commit(const reader_kv_cache &c, const __nv_bfloat16 *k_tree, con
                       const int32_t *path, const int32_t *n_acc, int max_path, int update_seq_lens, int32_t *slots,
                       int32_t *status, cudaStream_t st) {
     if (B <= 0) return;
-    kv_commit_kernel<<<B, 256, 0, st>>>(reinterpret_cast<__nv_bfloat16 *>(c.k_pool),
+    launch_pdl(kv_commit_kernel, dim3(B), dim3(256), 0, st, reinterpret_cast<__nv_bfloat16 *>(c.k_pool),
                                         reinterpret_cast<__nv_bfloat16 *>(c.v_pool), c.num_pages, c.n_kv_heads,
                                         c.head_dim, c.page_table, c.max_pages_per_seq, c.seq_lens,
                                         c.shared_prefix_len, k_tree, v_tree, T, path, n_acc, max_path,
