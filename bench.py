@@ -176,6 +176,25 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# N > 1: independent replicas (sequences do not interact), no data-path collective
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_tokens_per_s(batch, tree_nodes, world, steps, ms_max):
+    """Whole-job throughput: every rank verified batch * tree_nodes tokens per step; the job took the
+    time of its slowest rank."""
+    return batch * tree_nodes * world * steps / (ms_max * 1e-3)
+
+
+# ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -303,15 +322,13 @@ def run_ours(args):
     ms_e2e = f0.elapsed_time(f1)
 
     # ---- max over ranks
-    t = torch.tensor([ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel = t.tolist()
+    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel = max_over_ranks(
+        [ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel], dev, world)
 
     if rank == 0:
         tokens = B * T * world
-        value = tokens * K / (ms_total * 1e-3)
-        e2e = tokens * Ke / (ms_e2e * 1e-3)
+        value = aggregate_tokens_per_s(B, T, world, K, ms_total)
+        e2e = aggregate_tokens_per_s(B, T, world, Ke, ms_e2e)
         attn_bytes = w.attn_algorithmic_bytes()
         attn_flops = w.attn_algorithmic_flops()
         kernels = {
