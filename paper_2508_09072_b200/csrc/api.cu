@@ -188,7 +188,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.sched.seq_tile_start = reinterpret_cast<const int32_t *>(ws + w.seq_tile_start);
     p.sched.seq_ntiles = reinterpret_cast<const int32_t *>(ws + w.seq_ntiles);
     p.sched.seq_npages = reinterpret_cast<const int32_t *>(ws + w.seq_npages);
-    p.sched.units_per_seq = Hkv * n_mtiles;
+    p.sched.units_per_seq = Hkv;
     p.sched.n_mtiles = n_mtiles;
 
     const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);

@@ -38,8 +38,9 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
     if (d.b < 0) return;
     const int rows = min(kTileM, p.T * p.G - d.mt * kTileM);
     const bool has_cols = lane * 4 < D;
-    const int n_ctas = effective_ctas(p.sched.n_ctas, W);
-    const bool all_live = W >= n_ctas;   // with fewer tiles than CTAs some ranges are empty
+    const int nm = p.sched.n_mtiles;
+    const int n_lanes = effective_ctas(p.sched.n_ctas / nm, W);
+    const bool all_live = W >= n_lanes;   // with fewer tiles than CTAs some ranges are empty
 
     for (int rb = 0; rb < kRowsPerWarp; rb += kBatch) {
         const int r0 = warp * kRowsPerWarp + rb;
@@ -52,14 +53,15 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
             acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         // online merge over the CTAs c0 .. c_last, two slots x kBatch rows per round of loads
-        for (int cb = c0; cb <= d.c_last; cb += 2) {
+        // the unit's partials sit in the CTAs with the same M tile in the lanes c0 / nm .. c_last / nm
+        for (int cb = c0; cb <= d.c_last; cb += 2 * nm) {
             float2 ml[2][kBatch];
             float4 o[2][kBatch];
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
-                const int c = cb + k;
+                const int c = cb + k * nm;
                 // a CTA with an empty range wrote nothing
-                const bool live = c <= d.c_last && (all_live || range_begin(c + 1, n_ctas, W) != range_begin(c, n_ctas, W));
+                const bool live = c <= d.c_last && (all_live || range_begin(c / nm + 1, n_lanes, W) != range_begin(c / nm, n_lanes, W));
                 const int slot = c == c0 ? 2 * c + 1 : 2 * c;
 #pragma unroll
                 for (int q = 0; q < kBatch; ++q) {

@@ -18,19 +18,22 @@ constexpr int kMaxNodes = READER_MAX_NODES;
 //
 // A *unit* is (sequence b, KV head h, M tile mt): kTileM query rows (node j, group member g) with
 // row = j * G + g, attending over ntiles(b) KV tiles: the committed pages of b followed by the
-// tree tiles.  Units are ordered (b, h, mt), tiles within a unit in order, and the resulting flat
-// list of W tiles is cut into n_ctas contiguous ranges of near-equal length.  The part of a
-// range that lies in one unit is a *segment*.  A segment that covers its whole unit writes the
-// final output; any other segment writes an (m, l, O) partial into one of the CTA's two slots:
-// slot 2c when the segment does not start its unit, slot 2c+1 when it does.
+// tree tiles.  The KV streams (b, h), tiles in order, form one flat list of W tiles that is cut
+// into n_lanes contiguous ranges of near-equal length.  A *lane* is n_mtiles CTAs, one per M tile,
+// that walk the same range: CTA c has lane c / n_mtiles and M tile c % n_mtiles.  The CTAs of a
+// lane read the same K/V tiles at the same pace, so all but the first of them find the tile in
+// L2 (with an independent position per M tile every one of them fetched it from HBM again).
+// The part of a range that lies in one KV stream is a *segment*.  A segment that covers its whole
+// unit writes the final output; any other segment writes an (m, l, O) partial into one of the
+// CTA's two slots: slot 2c when the segment does not start its unit, slot 2c+1 when it does.
 // ---------------------------------------------------------------------------------------------
 struct Sched {
     const int32_t *seq_tile_start;  // [B+1] first flat tile of sequence b
     const int32_t *seq_ntiles;      // [B]   tiles per unit of sequence b (0: sequence skipped)
     const int32_t *seq_npages;      // [B]   committed pages among them
-    int32_t n_ctas;                 // CTAs launched; effective_ctas() of them share the work
-    int32_t units_per_seq;          // Hkv * n_mtiles
-    int32_t n_mtiles;
+    int32_t n_ctas;                 // CTAs launched (n_ctas / n_mtiles lanes); effective_ctas() of the lanes share the work
+    int32_t units_per_seq;          // KV streams per sequence: Hkv
+    int32_t n_mtiles;               // M tiles per KV stream = CTAs per lane
 };
 
 struct Segment {
@@ -73,8 +76,8 @@ __device__ __forceinline__ Segment segment_at(const Sched &s, int B, int cta, in
     int local = w - s.seq_tile_start[g.b];
     int unit = local / g.ntiles;
     g.tile_begin = local - unit * g.ntiles;
-    g.h = unit / s.n_mtiles;
-    g.mt = unit - g.h * s.n_mtiles;
+    g.h = unit;
+    g.mt = cta % s.n_mtiles;
     int left = range_end - w;
     g.tile_end = min(g.ntiles, g.tile_begin + left);
     g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
@@ -99,8 +102,8 @@ __device__ __forceinline__ Segment segment_at_warp(const Sched &s, int B, int ct
     int local = w - s.seq_tile_start[b];
     int unit = local / g.ntiles;
     g.tile_begin = local - unit * g.ntiles;
-    g.h = unit / s.n_mtiles;
-    g.mt = unit - g.h * s.n_mtiles;
+    g.h = unit;
+    g.mt = cta % s.n_mtiles;
     int left = range_end - w;
     g.tile_end = min(g.ntiles, g.tile_begin + left);
     g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
@@ -108,13 +111,27 @@ __device__ __forceinline__ Segment segment_at_warp(const Sched &s, int B, int ct
     return g;
 }
 
-// CTA whose range contains flat tile w.
+// Lane (of n_ctas lanes) whose range contains flat tile w.
 __device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
     int c = (int)(((int64_t)w * n_ctas) / W);
     if (c >= n_ctas) c = n_ctas - 1;
     while (c + 1 < n_ctas && range_begin(c + 1, n_ctas, W) <= w) ++c;
     while (c > 0 && range_begin(c, n_ctas, W) > w) --c;
     return c;
+}
+
+// The work of one CTA: its M tile and its lane's range of the flat tile list.
+struct CtaWork {
+    int mt, n_lanes, w_begin, w_end;
+};
+__device__ __forceinline__ CtaWork cta_work(const Sched &s, int cta, int W) {
+    CtaWork k;
+    const int lane = cta / s.n_mtiles;
+    k.mt = cta - lane * s.n_mtiles;
+    k.n_lanes = effective_ctas(s.n_ctas / s.n_mtiles, W);   // lanes that share the work
+    k.w_begin = range_begin(lane, k.n_lanes, W);           // a lane left without work gets W, W
+    k.w_end = range_begin(lane + 1, k.n_lanes, W);
+    return k;
 }
 
 // Written by the attention CTA that starts a unit it does not finish (at most one per CTA); read by
@@ -125,11 +142,11 @@ struct SplitDesc {
 
 // Called by one thread per segment: if the segment starts its unit without finishing it, note where
 // the unit's partials end so that the combine kernel can find them without any search.
-__device__ __forceinline__ void record_split(SplitDesc *desc, int n_ctas, const Segment &g, int cta, int w_seg_begin, int W) {
+__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, int n_lanes, const Segment &g, int cta, int w_seg_begin, int W) {
     if (g.tile_begin != 0 || g.full) return;
     SplitDesc d;
     d.b = g.b; d.h = g.h; d.mt = g.mt;
-    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, n_ctas, W);
+    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, n_lanes, W) * s.n_mtiles + g.mt;   // same M tile, last lane
     desc[cta] = d;
 }
 

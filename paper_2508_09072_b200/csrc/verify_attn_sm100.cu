@@ -236,9 +236,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     grid_dependency_wait();
     grid_launch_dependents();
     const int W = p.sched.seq_tile_start[p.B];
-    const int n_ctas = effective_ctas(p.sched.n_ctas, W);
-    const int w_begin = range_begin(cta, n_ctas, W);
-    const int w_end = range_begin(cta + 1, n_ctas, W);
+    const CtaWork cw = cta_work(p.sched, cta, W);
+    const int w_begin = cw.w_begin, w_end = cw.w_end;
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
@@ -399,7 +398,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         if (tid == 0) p.split_desc[cta].b = -1;
         while (w < w_end) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
-            if (tid == 0) record_split(p.split_desc, n_ctas, sg, cta, w, W);
+            if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, w, W);
             w += sg.tile_end - sg.tile_begin;
             const int L = p.seq_lens[sg.b];
             const int grow = sg.mt * kTileM + tid;
