@@ -374,6 +374,53 @@ def run_ours(args):
     rd.close()
 
 
+# ------------------------------------------------------------------------------------------------
+# tree-size sweep: T_V(T), the verification-attention time as a function of the draft-tree size
+# (Sec. 3.2: reads grow with s + gamma, FLOPs with gamma (s + gamma); Theorem 1 needs T_V(T))
+# ------------------------------------------------------------------------------------------------
+def run_sweep(args):
+    import numpy as np
+    import torch
+    from paper_2508_09072_b200 import binding, workloads as W
+    torch.cuda.set_device(0)
+    rd = binding.Reader(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    peaks, _ = load_peaks()
+    rows = []
+    for B in (1, 8, 32):
+        for T in (8, 16, 32, 64, 128):
+            rng = np.random.default_rng(77 + B)
+            lens = rng.integers(1024, 4097, size=B)
+            w = W.build_workload(f"sweep-b{B}-t{T}", 9000 + 131 * B + T, lens, T, 32, 8, 128,
+                                 lambda r: W.capped_recursive_tree(r, T, 12, 4), max_path=12, vocab=16,
+                                 shuffle_pages=True, with_logits=False)
+            d = binding.to_device(w, with_logits=False)
+            anc, _, _ = rd.tree_encode(d.parent)
+            out = torch.empty_like(d.q)
+            st = torch.empty(B, dtype=torch.int32, device="cuda")
+            ws = rd.workspace(B, T, 32, 8, 128)
+            call = lambda: rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out,
+                                          status=st, workspace=ws)
+            for _ in range(3):
+                call()
+            ts = []
+            for _ in range(args.sweep_iters):
+                flush.zero_()                                  # cold L2: the small cases fit in it
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); call(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ts.sort()
+            us = ts[len(ts) // 2] * 1e3
+            t_hbm = w.attn_algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6
+            t_tc = w.attn_algorithmic_flops() / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+            rows.append({"batch": B, "tree_nodes": T, "committed_tokens": int(lens.sum()), "call_us": us,
+                         "tokens_per_s": B * T / (us * 1e-6), "t_hbm_us": t_hbm, "t_tensor_us": t_tc,
+                         "bound": "hbm" if t_hbm >= t_tc else "tensor"})
+    print(json.dumps({"sweep": "verify-attention call time vs draft-tree size (cold L2, median)", "rows": rows}))
+    rd.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -384,8 +431,12 @@ def main():
     ap.add_argument("--kernel", type=int, default=0, help="attention kernel: 0 auto, 1 CUDA-core, 2 tensor-core")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-tree", action="store_true", help="measure the attention call for several tree sizes instead")
+    ap.add_argument("--sweep-iters", type=int, default=15)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep_tree:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
