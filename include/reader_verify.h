@@ -27,6 +27,8 @@
  *     outside the pool, a length beyond the page table.  A sequence with a non-zero status gets
  *     defined outputs (attention rows and lse zero; n_acc 0, path -1, bonus -1; nothing
  *     committed) and does not disturb the others.  No kernel traps, asserts or waits unbounded.
+ *   - An empty batch (batch = 0) is legal everywhere: the call returns READER_OK, launches nothing
+ *     and looks at no tensor pointer.
  *   - Tree convention: node 0 is the root = the last token already chosen by the target model
  *     (its K/V is part of the tree tensors, not yet of the cache); parent[0] = -1 and
  *     0 <= parent[j] < j.  At most READER_MAX_NODES nodes.

@@ -61,8 +61,9 @@ extern "C" reader_status reader_accept_noalloc(reader_ctx *ctx, const reader_tre
                                                int32_t max_path, int32_t *path_out, int32_t *n_acc_out,
                                                int32_t *bonus_out, int32_t *status_out, void *stream) {
     using namespace reader;
-    if (!ctx || !tree || !tree->parent || !node_tokens || !logits || !target_ids || !path_out || !n_acc_out ||
-        !bonus_out || !status_out)
+    if (!ctx || !tree) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;
+    if (!tree->parent || !node_tokens || !logits || !target_ids || !path_out || !n_acc_out || !bonus_out || !status_out)
         return READER_ERR_INVALID_ARG;
     const int B = tree->batch, T = tree->n_nodes;
     if (B < 0 || T < 1 || T > kMaxNodes || max_path < 1 || vocab < 1 ||

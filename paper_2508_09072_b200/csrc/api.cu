@@ -137,8 +137,9 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
                                  const void *v_tree, const reader_kv_cache *cache, const reader_tree *tree,
                                  float softmax_scale, void *out, float *lse_out, void *workspace,
                                  size_t workspace_bytes, int32_t *status_out, void *stream) {
-    if (!ctx || !q || !k_tree || !v_tree || !cache || !tree || !out || !workspace || !status_out)
-        return READER_ERR_INVALID_ARG;
+    if (!ctx || !cache || !tree) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;   // an empty batch has no tensors to point at
+    if (!q || !k_tree || !v_tree || !out || !workspace || !status_out) return READER_ERR_INVALID_ARG;
     const int B = tree->batch, T = tree->n_nodes, Hq = n_q_heads, Hkv = cache->n_kv_heads, D = cache->head_dim;
     if (!cache->k_pool || !cache->v_pool || !cache->page_table || !cache->seq_lens || !tree->parent)
         return READER_ERR_INVALID_ARG;
@@ -215,8 +216,9 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
                             const float *logits, int32_t vocab, int32_t *target_ids, int32_t max_path,
                             int32_t *path_out, int32_t *n_acc_out, int32_t *bonus_out, void *workspace,
                             size_t workspace_bytes, int32_t *status_out, void *stream) {
-    if (!ctx || !tree || !tree->parent || !node_tokens || !target_ids || !path_out || !n_acc_out || !bonus_out ||
-        !status_out)
+    if (!ctx || !tree) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;
+    if (!tree->parent || !node_tokens || !target_ids || !path_out || !n_acc_out || !bonus_out || !status_out)
         return READER_ERR_INVALID_ARG;
     const int B = tree->batch, T = tree->n_nodes;
     if (B < 0 || T < 1 || T > kMaxNodes || max_path < 1) return READER_ERR_INVALID_ARG;
@@ -252,7 +254,9 @@ reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const vo
                                int32_t batch, int32_t n_nodes, const int32_t *path, const int32_t *n_acc,
                                int32_t max_path, int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out,
                                void *stream) {
-    if (!ctx || !cache || !k_tree || !v_tree || !path || !n_acc || !slots_out || !status_out ||
+    if (!ctx || !cache) return READER_ERR_INVALID_ARG;
+    if (batch == 0) return READER_OK;
+    if (!k_tree || !v_tree || !path || !n_acc || !slots_out || !status_out ||
         !cache->k_pool || !cache->v_pool || !cache->page_table || !cache->seq_lens)
         return READER_ERR_INVALID_ARG;
     if (batch < 0 || n_nodes < 1 || n_nodes > kMaxNodes || max_path < 1 || cache->n_kv_heads < 1 ||

@@ -139,6 +139,40 @@ def test_attn_shapes_and_ragged_lengths(rd, case, kernel):
     check_attn(w, got, status, lse)
 
 
+def test_attn_random_shapes(rd):
+    """Seeded random shapes: tree size, GQA group (1..16, so 1 to 16 M tiles per KV stream), head
+    dimension, batch and ragged committed lengths (empty caches and exact page multiples included)."""
+    rng = np.random.default_rng(20250809)
+    for case in range(28):
+        T = int(rng.choice([1, 2, 3, 7, 16, 31, 32, 33, 63, 64, 65, 100, 127, 128]))
+        G = int(rng.choice([1, 2, 4, 8, 16]))
+        Hkv = int(rng.choice([1, 2, 3]))
+        D = int(rng.choice([64, 128]))
+        B = int(rng.integers(1, 6))
+        lens = [int(x) for x in rng.choice([0, 1, 5, 63, 64, 65, 127, 128, 129, 200, 333, 640], size=B)]
+        w = W.build_workload("r", 5000 + case, lens, T, G * Hkv, Hkv, D,
+                             lambda r: W.capped_recursive_tree(r, T, 12, 4) if T > 1 else np.array([-1], np.int32),
+                             max_path=12, vocab=16, shuffle_pages=True, with_logits=False, spare_pages=2)
+        got, status, lse = gpu_attn(rd, w, kernel=0, pre_encode=bool(case & 1))
+        try:
+            check_attn(w, got, status, lse)
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: T={T} G={G} Hkv={Hkv} D={D} lens={lens}: {e}")
+
+
+def test_attn_empty_batch_is_a_no_op(rd):
+    from paper_2508_09072_b200 import binding
+    w = W.make("c1", with_logits=False)
+    d = binding.to_device(w, with_logits=False)
+    empty = lambda t: t[:0].contiguous()
+    cache = binding.KvCache(d.cache.k_pool, d.cache.v_pool, empty(d.cache.page_table).reshape(0, d.cache.page_table.shape[1]),
+                            empty(d.cache.seq_lens))
+    out, status = rd.verify_attn(empty(d.q), empty(d.k_tree), empty(d.v_tree), cache, empty(d.parent), w.scale,
+                                 workspace=rd.workspace(1, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim))
+    torch.cuda.synchronize()
+    assert out.shape[0] == 0 and status.shape[0] == 0
+
+
 def test_attn_many_short_sequences_and_widened_trees(rd):
     rng = np.random.default_rng(77)
     lens = rng.integers(0, 200, size=40)
