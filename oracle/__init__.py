@@ -49,6 +49,7 @@ def _load():
                                            p32, c_int, p32, p32, c_int, c_int, c_int, c_double,
                                            pd, c_void_p, c_void_p, c_int64, p32]
         lib.oracle_argmax.argtypes = [pf, c_int64, c_int64, p32]
+        lib.oracle_sample_targets.argtypes = [pf, p32, pf, c_int, c_int, c_int64, c_double, p32]
         lib.oracle_accept.argtypes = [p32, p32, p32, c_int, c_int, c_int, p32, p32, p32, p32]
         lib.oracle_kv_commit.argtypes = [p16, p16, c_int, c_int, c_int, c_int, p32, c_int, p32, c_int,
                                          p16, p16, c_int, c_int, p32, p32, c_int, c_int, p32, p32]
@@ -137,6 +138,19 @@ def argmax(logits) -> np.ndarray:
     out = np.zeros(rows, dtype=np.int32)
     _load().oracle_argmax(_ptr(logits, c_float), rows, V, _ptr(out, c_int32))
     return out.reshape(logits.shape[:-1])
+
+
+def sample_targets(logits, parent, uniforms, temperature: float) -> np.ndarray:
+    """Appendix C, randomized policy: per-node target id x* = F(P, U) by temperature inverse-CDF
+    sampling; uniforms f32 [B, T], entry level-1 serves all nodes of that tree level."""
+    logits, parent, uniforms = _c(logits, np.float32), _c(parent, np.int32), _c(uniforms, np.float32)
+    B, T = parent.shape
+    V = logits.shape[-1]
+    assert logits.shape == (B, T, V) and uniforms.shape == (B, T)
+    out = np.zeros((B, T), dtype=np.int32)
+    _load().oracle_sample_targets(_ptr(logits, c_float), _ptr(parent, c_int32), _ptr(uniforms, c_float), B, T, V,
+                                  float(temperature), _ptr(out, c_int32))
+    return out
 
 
 def accept(parent, node_tokens, target_ids, max_path: int):

@@ -17,6 +17,8 @@
  *   oracle_accept           invariants 1-3 and the deterministic theorem:
  *                           compare the base model's greedy choice with the
  *                           drafted tokens, keep the longest consistent prefix.
+ *   oracle_sample_targets   Appendix C, randomized decoding: x* = F(P, U_t) with
+ *                           coupled uniforms, temperature inverse-CDF sampling.
  *   oracle_kv_commit        Sec. 4.3 and Algorithm 4 (KVCacheRearrange): the
  *                           accepted entries are concatenated tightly behind
  *                           the committed cache, per sample.
@@ -256,6 +258,74 @@ void oracle_argmax(const float *logits, int64_t rows, int64_t vocab, int32_t *ta
  * lowest e among equals.  bonus = target[e] is the token invariant 3 commits
  * after the last accepted one.  path is padded with -1.
  */
+/*
+ * Randomized policy of Appendix C ("Randomized decoding"): x* = F(P_theta(. | prefix), U_t), one
+ * uniform U_t per output POSITION, shared by the base run and the verifier.  Every node at tree
+ * level lv (root = 1) proposes a token for position lv, and its target is the token the policy emits
+ * for position lv + 1: all nodes of one level therefore use the same uniform, u[b][lv - 1].
+ *
+ * F is temperature sampling by inverse CDF, stated so that a float never decides the token by a
+ * rounding that depends on summation order:
+ *   c    = (float)(log2(e) / temperature)                 (double division, rounded once)
+ *   m    = row maximum (NaN never wins; NaN in slot 0 counts as -inf)
+ *   x_v  = (l_v - m) * c          two fp32 operations; NaN or x_v < -64 gives weight 0
+ *   n    = nearest integer to x_v (ties to even), f = x_v - n in [-1/2, 1/2]
+ *   p    = 1 + f(c1 + f(c2 + f(c3 + f(c4 + f c5))))      fp32 Horner with fused multiply-adds,
+ *          c_k = ln(2)^k / k! rounded to fp32            (2^f to about 3e-6)
+ *   W_v  = trunc(p * 2^(n + 40))                          integer weight, at most 2^40
+ *   S    = sum_v W_v (exact, 64-bit);  U = trunc(u * 2^24);  thr = (S * U) >> 24 (exact, 128-bit)
+ *   x*   = the first v whose inclusive prefix sum of W exceeds thr      (0 if S = 0)
+ * Ties on "measure-zero boundaries" are thus resolved towards the lower token id.
+ */
+static uint64_t sample_weight(float l, float m, float c)
+{
+    const float x = (l - m) * c;
+    if (!(x >= -64.0f)) return 0;                 /* also catches NaN */
+    const float n = nearbyintf(x);                /* default rounding mode: ties to even */
+    const float f = x - n;
+    float p = 1.3333558146e-3f;
+    p = fmaf(p, f, 9.6181291076e-3f);
+    p = fmaf(p, f, 5.5504108665e-2f);
+    p = fmaf(p, f, 2.4022650696e-1f);
+    p = fmaf(p, f, 6.9314718056e-1f);
+    p = fmaf(p, f, 1.0f);
+    return (uint64_t)ldexpf(p, (int)n + 40);      /* exact scaling, then truncation */
+}
+
+int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double temperature)
+{
+    const float c = (float)(1.4426950408889634 / temperature);
+    float m = row[0];
+    if (isnan(m)) m = -INFINITY;
+    for (int64_t v = 1; v < vocab; ++v)
+        if (row[v] > m) m = row[v];
+    if (m == -INFINITY) return 0;                 /* nothing has weight */
+    uint64_t total = 0;
+    for (int64_t v = 0; v < vocab; ++v) total += sample_weight(row[v], m, c);
+    if (total == 0) return 0;
+    const uint64_t U = (uint64_t)(u * 16777216.0f);          /* u in [0, 1): 24 bits */
+    const uint64_t thr = (uint64_t)(((unsigned __int128)total * U) >> 24);
+    uint64_t run = 0;
+    for (int64_t v = 0; v < vocab; ++v) {
+        run += sample_weight(row[v], m, c);
+        if (run > thr) return (int32_t)v;
+    }
+    return (int32_t)(vocab - 1);                  /* not reached: thr < total */
+}
+
+/* target[b][j] for every node; uniforms f32 [B][T], entry lv - 1 serves the nodes of level lv. */
+void oracle_sample_targets(const float *logits, const int32_t *parent, const float *uniforms,
+                           int B, int T, int64_t vocab, double temperature, int32_t *target)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < (int64_t)B * T; ++r) {
+        const int b = (int)(r / T), j = (int)(r % T);
+        int lv = 0;
+        for (int i = j, steps = 0; i >= 0 && steps < T; i = parent[(size_t)b * T + i], ++steps) ++lv;
+        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature);
+    }
+}
+
 void oracle_accept(const int32_t *parent, const int32_t *tok, const int32_t *target,
                    int batch, int n_nodes, int max_path,
                    int32_t *path, int32_t *n_acc, int32_t *bonus, int32_t *status)

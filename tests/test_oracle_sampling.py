@@ -1,0 +1,115 @@
+"""Pins for the oracle's randomized policy (Appendix C: x* = F(P, U_t) with coupled uniforms).
+
+None of these retypes the sampler's arithmetic: they check it against closed forms, against the
+softmax distribution it must realise, against structural facts (monotone in u, one uniform per
+tree level) and against the randomized-losslessness theorem on a toy model.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2508_09072_b200 import workloads as W
+
+
+def one_row(logits, u, temperature=1.0):
+    lg = np.asarray(logits, np.float32).reshape(1, 1, -1)
+    return int(oracle.sample_targets(lg, np.array([[-1]], np.int32), np.array([[u]], np.float32), temperature)[0, 0])
+
+
+def test_equal_logits_give_the_floor_of_u_times_vocab():
+    for V in (2, 8, 1000):
+        for u in (0.0, 0.1249, 0.125, 0.5, 0.777, 0.999999):
+            assert one_row(np.zeros(V), u) == int(np.float32(u) * V), (V, u)
+            assert one_row(np.full(V, -3.25), u, temperature=0.3) == int(np.float32(u) * V)
+
+
+def test_frequencies_over_a_grid_of_uniforms_are_the_softmax():
+    rng = np.random.default_rng(1)
+    for temperature in (0.5, 1.0, 2.0):
+        lg = rng.standard_normal(6).astype(np.float32) * 2
+        n = 1 << 14
+        us = (np.arange(n, dtype=np.float64) + 0.5) / n
+        got = np.bincount([one_row(lg, u, temperature) for u in us], minlength=6) / n
+        z = lg.astype(np.float64) / temperature
+        p = np.exp(z - z.max()); p /= p.sum()
+        assert np.abs(got - p).max() <= 1.0 / n + 2e-5, (temperature, got, p)     # grid step + 2^f polynomial
+        # inverse CDF: the chosen token never decreases as u grows
+        picks = [one_row(lg, u, temperature) for u in np.linspace(0, 0.999, 400)]
+        assert picks == sorted(picks)
+
+
+def test_low_temperature_is_greedy_and_u_zero_picks_the_first_token_with_weight():
+    rng = np.random.default_rng(2)
+    lg = rng.standard_normal(50).astype(np.float32)
+    for u in (0.0, 0.3, 0.9):
+        assert one_row(lg, u, temperature=1e-3) == int(np.argmax(lg))
+    lg2 = np.array([-np.inf, np.nan, -200.0, 1.0, 2.0], np.float32)
+    assert one_row(lg2, 0.0) == 3                      # -inf, NaN and a weight below 2^-64 are never drawn
+    assert one_row(np.array([np.nan, np.nan], np.float32), 0.5) == 0
+    assert one_row(np.array([-np.inf, -np.inf], np.float32), 0.5) == 0
+
+
+def test_one_uniform_per_tree_level():
+    """Siblings (and cousins) propose tokens for the same position, so they share their uniform;
+    the uniform a node uses is entry level-1 of its sequence's row."""
+    rng = np.random.default_rng(3)
+    T, V = 7, 40
+    parent = np.array([[-1, 0, 0, 1, 1, 2, 5]], np.int32)     # levels 1 2 2 3 3 3 4
+    row = rng.standard_normal(V).astype(np.float32)
+    logits = np.tile(row, (1, T, 1))
+    u = rng.random((1, T)).astype(np.float32)
+    tgt = oracle.sample_targets(logits, parent, u, 1.0)[0]
+    lv = oracle.levels(parent[0])
+    for j in range(T):
+        assert tgt[j] == one_row(row, u[0, lv[j] - 1])
+    assert tgt[1] == tgt[2] and tgt[3] == tgt[4] == tgt[5]
+
+
+def toy_logits(prefix, V):
+    """A deterministic stand-in for the target model: logits are a hash-seeded function of the prefix."""
+    seed = 1469598103934665603
+    for t in prefix:
+        seed = ((seed ^ int(t)) * 1099511628211) % (1 << 64)
+    return np.random.default_rng(seed).standard_normal(V).astype(np.float32) * 1.5
+
+
+def test_randomized_losslessness_with_coupled_uniforms():
+    """Appendix C, randomized theorem: READER with draft trees, verified against the sampled token
+    x*_t = F(P(. | prefix), U_t) and coupled to the same uniforms, emits exactly the base run."""
+    V, steps, temperature = 12, 40, 0.8
+    rng = np.random.default_rng(7)
+    U = rng.random(steps + 16).astype(np.float32)
+    base = [3]
+    while len(base) < steps + 1:
+        t = len(base)                                           # position of the token to draw
+        base.append(one_row(toy_logits(base, V), U[t], temperature))
+    out, n_steps = [3], 0
+    while len(out) < steps + 1:
+        T = 10
+        parent = W.capped_recursive_tree(rng, T, 5, 3)
+        lv = oracle.levels(parent)
+        tok = rng.integers(0, V, size=T).astype(np.int32)
+        tok[0] = out[-1]
+        for j in range(1, T):                                   # plant the true continuation on some branches
+            if rng.random() < 0.6:
+                pre, i = [], j
+                while parent[i] >= 0:
+                    i = parent[i]; pre.append(tok[i])
+                prefix = out[:-1] + pre[::-1]
+                tok[j] = one_row(toy_logits(prefix, V), U[len(prefix)], temperature)
+        logits = np.zeros((1, T, V), np.float32)
+        for j in range(T):
+            pre, i = [tok[j]], j
+            while parent[i] >= 0:
+                i = parent[i]; pre.append(tok[i])
+            logits[0, j] = toy_logits(out[:-1] + pre[::-1], V)
+        pos0 = len(out)                                         # position of the token after the root
+        u_rows = np.zeros((1, T), np.float32)
+        u_rows[0, : T] = U[pos0: pos0 + T]
+        tgt = oracle.sample_targets(logits, parent[None], u_rows, temperature)
+        a = oracle.accept(parent[None], tok[None], tgt, T)
+        path = a["path"][0][: a["n_acc"][0]]
+        out += [int(tok[j]) for j in path[1:]] + [int(a["bonus"][0])]
+        n_steps += 1
+    assert out[: steps + 1] == base[: steps + 1]
+    assert n_steps < steps                                       # several tokens per step were accepted
