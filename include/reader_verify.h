@@ -168,6 +168,25 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
                             int32_t *status_out, void *stream);
 
 /*
+ * Appendix C, randomized decoding: the per-node target of a sampling policy, x* = F(P, U_t), for
+ * use as `target_ids` of reader_accept(logits = NULL).  F is temperature sampling through the
+ * inverse CDF.  One uniform serves one output position: every node of tree level lv (root = 1)
+ * uses uniforms[b][lv - 1], and the caller passes the same uniforms the plain (non-speculative) run
+ * would use for those positions -- that coupling is what makes the decoded text identical.
+ *   logits      f32 [batch][n_nodes][vocab], 16-byte aligned
+ *   uniforms    f32 [batch][n_nodes], values in [0, 1) (clamped into it)
+ *   temperature > 0
+ *   target_ids  i32 [batch][n_nodes] out
+ * The CDF is integer arithmetic (fp32 weights from a fixed fused-multiply-add polynomial for
+ * 2^x, truncated to 40 fractional bits; exact 64-bit sums; threshold (S * trunc(u 2^24)) >> 24;
+ * first token whose inclusive prefix sum exceeds it), so the result does not depend on how the
+ * sum is parallelised.  NaN and -inf logits are never drawn; a row without any weight gives 0.
+ * vocab <= 2 Mi.  No workspace.
+ */
+reader_status reader_sample_targets(reader_ctx *ctx, const reader_tree *tree, const float *logits, int32_t vocab,
+                                    const float *uniforms, float temperature, int32_t *target_ids, void *stream);
+
+/*
  * Sec. 4.3 / Algorithm 4 in per-step form.  For k < n_acc[b] the K/V rows of node path[b][k]
  * (all KV heads) are copied to logical position seq_lens[b] + k of sequence b, i.e. pool slot
  * page_table[b][(L+k)/page_size]*page_size + (L+k)%page_size, which is also written to

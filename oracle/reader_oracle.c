@@ -303,7 +303,9 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
     uint64_t total = 0;
     for (int64_t v = 0; v < vocab; ++v) total += sample_weight(row[v], m, c);
     if (total == 0) return 0;
-    const uint64_t U = (uint64_t)(u * 16777216.0f);          /* u in [0, 1): 24 bits */
+    if (!(u >= 0.0f)) u = 0.0f;                              /* u is meant to lie in [0, 1) */
+    if (u > 0.99999994f) u = 0.99999994f;
+    const uint64_t U = (uint64_t)(u * 16777216.0f);          /* 24 bits */
     const uint64_t thr = (uint64_t)(((unsigned __int128)total * U) >> 24);
     uint64_t run = 0;
     for (int64_t v = 0; v < vocab; ++v) {
@@ -321,7 +323,11 @@ void oracle_sample_targets(const float *logits, const int32_t *parent, const flo
     for (int64_t r = 0; r < (int64_t)B * T; ++r) {
         const int b = (int)(r / T), j = (int)(r % T);
         int lv = 0;
-        for (int i = j, steps = 0; i >= 0 && steps < T; i = parent[(size_t)b * T + i], ++steps) ++lv;
+        for (int i = j, steps = 0; i >= 0 && i < T && steps < T; ++steps) {
+            ++lv;
+            const int up = parent[(size_t)b * T + i];
+            i = up < i ? up : -1;                 /* a malformed array cannot send the walk astray */
+        }
         target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature);
     }
 }

@@ -25,7 +25,7 @@ NOALLOC_MAX_ROWS = 4096
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
            "reader_set_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
-           "reader_kv_commit", "reader_accept_noalloc")
+           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets")
 
 
 class ReaderError(RuntimeError):
@@ -79,6 +79,8 @@ def load_library() -> ctypes.CDLL:
     lib.reader_accept_noalloc.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.reader_accept_noalloc.restype = c_int32
+    lib.reader_sample_targets.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_int32, c_void_p, c_float, c_void_p, c_void_p]
+    lib.reader_sample_targets.restype = c_int32
     lib.reader_kv_commit.argtypes = [c_void_p, POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
     lib.reader_kv_commit.restype = c_int32
@@ -264,6 +266,21 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_accept_noalloc")
         return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
+
+    def sample_targets(self, parent: torch.Tensor, logits: torch.Tensor, uniforms: torch.Tensor, temperature: float,
+                       target_ids: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """reader_sample_targets: per-node target ids of the temperature-sampling policy with one coupled
+        uniform per tree level (feed the result to accept(target_ids=...))."""
+        _dev(parent, torch.int32, "parent"); _dev(logits, torch.float32, "logits"); _dev(uniforms, torch.float32, "uniforms")
+        B, T = parent.shape
+        if target_ids is None:
+            target_ids = torch.empty((B, T), dtype=torch.int32, device=parent.device)
+        tree = _Tree(B, T, parent.data_ptr(), None)
+        st = self.lib.reader_sample_targets(self._h, ctypes.byref(tree), _ptr(logits), logits.shape[-1], _ptr(uniforms),
+                                            float(temperature), _ptr(target_ids), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_sample_targets")
+        return target_ids
 
     def kv_commit(self, cache: KvCache, k_tree: torch.Tensor, v_tree: torch.Tensor, path: torch.Tensor,
                   n_acc: torch.Tensor, update_seq_lens: bool = True, slots: Optional[torch.Tensor] = None,

@@ -1,0 +1,92 @@
+"""GPU parity of reader_sample_targets (Appendix C, randomized policy) against the oracle: the
+CDF is integer arithmetic on both sides, so every target id must match exactly."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2508_09072_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rd():
+    from paper_2508_09072_b200 import binding
+    r = binding.Reader(0)
+    yield r
+    r.close()
+
+
+def gpu_sample(rd, parent, logits, uniforms, temperature):
+    t = rd.sample_targets(torch.from_numpy(parent).cuda(), torch.from_numpy(logits).cuda(),
+                          torch.from_numpy(uniforms).cuda(), temperature)
+    torch.cuda.synchronize()
+    return t.cpu().numpy()
+
+
+@pytest.mark.parametrize("vocab", [1, 2, 7, 64, 1000, 2048, 2049, 4099, 50024])
+@pytest.mark.parametrize("temperature", [0.25, 1.0, 1.7])
+def test_sample_targets_match_the_oracle(rd, vocab, temperature):
+    rng = np.random.default_rng(vocab * 7 + int(temperature * 100))
+    B, T = 3, 21
+    parent = np.stack([W.capped_recursive_tree(rng, T, 7, 3), W.chain_tree(T), W.star_tree(T)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, vocab)) * 3).astype(np.float32)
+    u = rng.random((B, T)).astype(np.float32)
+    u[0, 0], u[1, 1], u[2, 1] = 0.0, 0.99999994, 0.5
+    if vocab >= 7:
+        logits[0, 1, :] = 0.0                       # ties everywhere
+        logits[0, 2, 3] = np.nan
+        logits[0, 3, :] = -np.inf
+        logits[0, 4, :] = np.nan
+        logits[1, 2, : vocab // 2] = -np.inf
+        logits[1, 3, vocab - 1] = 80.0              # one dominant token at the end
+        logits[2, 5, 0] = np.inf
+    got = gpu_sample(rd, parent, logits, u, temperature)
+    ref = oracle.sample_targets(logits, parent, u, temperature)
+    np.testing.assert_array_equal(got, ref)
+
+
+def test_sample_targets_full_vocabulary_and_out_of_range_uniforms(rd):
+    rng = np.random.default_rng(5)
+    B, T, V = 2, 32, 128256
+    parent = np.stack([W.capped_recursive_tree(rng, T, 6, 4) for _ in range(B)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, V)) * 2).astype(np.float32)
+    u = rng.random((B, T)).astype(np.float32)
+    u[0, 2], u[0, 3], u[1, 0] = -0.5, 1.5, np.nan       # clamped into [0, 1)
+    got = gpu_sample(rd, parent, logits, u, 0.9)
+    ref = oracle.sample_targets(logits, parent, u, 0.9)
+    np.testing.assert_array_equal(got, ref)
+    assert len(set(got[0].tolist())) > 1
+
+
+def test_sampled_policy_step_matches_oracle_step(rd):
+    """sample targets -> accept (given targets) -> commit, against the same three oracle calls."""
+    from paper_2508_09072_b200 import binding
+    w = W.make("c3", reduced=True)
+    rng = np.random.default_rng(11)
+    u = rng.random((w.batch, w.n_nodes)).astype(np.float32)
+    d = binding.to_device(w)
+    tgt = rd.sample_targets(d.parent, d.logits, torch.from_numpy(u).cuda(), 0.7)
+    acc = rd.accept(d.parent, d.node_tokens, w.max_path, target_ids=tgt)
+    slots, _ = rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc["path"], acc["n_acc"])
+    torch.cuda.synchronize()
+    rt = oracle.sample_targets(w.logits, w.parent, u, 0.7)
+    ra = oracle.accept(w.parent, w.node_tokens, rt, w.max_path)
+    rc = oracle.kv_commit(w.k_pool, w.v_pool, w.page_table, w.seq_lens, 0, w.k_tree, w.v_tree, ra["path"], ra["n_acc"])
+    np.testing.assert_array_equal(tgt.cpu().numpy(), rt)
+    for k in ("path", "n_acc", "bonus"):
+        np.testing.assert_array_equal(acc[k].cpu().numpy(), ra[k], err_msg=k)
+    np.testing.assert_array_equal(slots.cpu().numpy(), rc["slots"])
+    np.testing.assert_array_equal(binding.bf16_bits(d.cache.k_pool), rc["k_pool"])
+
+
+def test_sample_targets_argument_errors(rd):
+    from paper_2508_09072_b200 import binding
+    parent = torch.from_numpy(W.chain_tree(4)[None]).cuda()
+    logits = torch.zeros((1, 4, 8), dtype=torch.float32, device="cuda")
+    u = torch.zeros((1, 4), dtype=torch.float32, device="cuda")
+    for bad_t in (0.0, -1.0, float("nan")):
+        with pytest.raises(binding.ReaderError) as e:
+            rd.sample_targets(parent, logits, u, bad_t)
+        assert e.value.code == binding.ERR_INVALID_ARG
