@@ -288,6 +288,19 @@ def run_ours(args):
     t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / Kb
     t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
 
+    # ---- the sampling policy's target kernel (an alternative to the argmax; not part of the step)
+    uni = torch.rand((B, T), dtype=torch.float32, device=dev)
+    tgt_s = torch.empty((B, T), dtype=torch.int32, device=dev)
+    for _ in range(3):
+        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s)
+    s0, s1 = mk(), mk()
+    s0.record()
+    for _ in range(20):
+        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s)
+    s1.record()
+    barrier()
+    t_sample = s0.elapsed_time(s1) / 20
+
     # ---- end to end: host buffers in, results out, every step
     host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits")}
     host_out = {"out": torch.empty(out.shape, dtype=out.dtype).pin_memory(),
@@ -339,6 +352,9 @@ def run_ours(args):
             "accept": {"call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
                        "gbs": w.logits_bytes() / (t_accept * 1e-3) / 1e9},
             "kv_commit": {"call_ms": t_commit},
+            "sample_targets": {"call_ms": t_sample, "algorithmic_bytes": w.logits_bytes(),
+                               "gbs": w.logits_bytes() / (t_sample * 1e-3) / 1e9,
+                               "note": "sampling policy (Appendix C); replaces the argmax when used; not in the step"},
         }
         t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
         t_tc = attn_flops / (peaks["bf16_tflops_sustained"] * 1e12)

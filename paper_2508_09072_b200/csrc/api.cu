@@ -261,7 +261,7 @@ reader_status reader_sample_targets(reader_ctx *ctx, const reader_tree *tree, co
     if (vocab > sample_max_vocab()) return READER_ERR_UNSUPPORTED;
     if (reader_status st = check_device(ctx)) return st;
     const float c = (float)(1.4426950408889634 / (double)temperature);
-    launch_sample(logits, (int64_t)B * T, vocab, tree->parent, uniforms, T, c, target_ids, (cudaStream_t)stream);
+    launch_sample(logits, (int64_t)B * T, vocab, tree->parent, uniforms, T, c, target_ids, ctx->n_sm, (cudaStream_t)stream);
     return launch_status();
 }
 

@@ -11,29 +11,40 @@
 //       c_k = ln(2)^k / k! in fp32
 //   W_v = trunc(p * 2^(n + 40));  S = sum W_v;  U = trunc(u * 2^24);  thr = (S * U) >> 24
 //   x*  = first v whose inclusive prefix sum of W exceeds thr (0 when S = 0)
-// One CTA per row: warps take tiles of 2048 logits (coalesced 16-byte loads), tile sums go to
-// shared memory, the tile holding the crossing is scanned in element order by one warp.
+// One CTA of 256 threads per row (four resident per SM; a grid-stride loop covers very large
+// batches).  A row needs two passes, maximum then weights; both come from HBM, which is what bounds
+// the kernel (2 x 4 bytes per logit at ~4.7 TB/s).  Warps take tiles of 2048 logits (coalesced
+// 16-byte loads), tile sums go to shared memory, the tile holding the crossing is scanned in
+// element order by one warp.
 #include "common.cuh"
 
 namespace reader {
 
-constexpr int kSampleThreads = 512;
+constexpr int kSampleThreads = 256;
 constexpr int kSampleTile = 2048;
 constexpr int kSampleMaxTiles = 1024;   // vocabularies up to 2 Mi entries
 
+// The weight of the definition above, computed without conversion instructions (they run on the slow
+// special-function pipe): adding 1.5 * 2^23 rounds x to the nearest integer, ties to even, and leaves
+// that integer in the low mantissa bits; trunc(p * 2^(n + 40)) is a shift of p's 24-bit significand.
 __device__ __forceinline__ unsigned long long sample_weight(float l, float m, float c) {
     const float x = __fmul_rn(__fsub_rn(l, m), c);
-    if (!(x >= -64.0f)) return 0ull;
-    const float n = rintf(x);
+    if (!(x >= -64.0f)) return 0ull;                                  // also NaN
+    const float magic = 12582912.0f;                                   // 1.5 * 2^23
+    const float shifted = __fadd_rn(x, magic);
+    const float n = __fsub_rn(shifted, magic);                         // rint(x), exact for |x| <= 64
+    const int ni = __float_as_int(shifted) - 0x4B400000;               // the same integer
     const float f = __fsub_rn(x, n);
     float p = 1.3333558146e-3f;
     p = __fmaf_rn(p, f, 9.6181291076e-3f);
     p = __fmaf_rn(p, f, 5.5504108665e-2f);
     p = __fmaf_rn(p, f, 2.4022650696e-1f);
     p = __fmaf_rn(p, f, 6.9314718056e-1f);
-    p = __fmaf_rn(p, f, 1.0f);
-    const float scale = __int_as_float(((int)n + 40 + 127) << 23);   // 2^(n + 40), exponent in [-24, 40]
-    return __float2ull_rz(__fmul_rn(p, scale));                      // exact product, then truncation
+    p = __fmaf_rn(p, f, 1.0f);                                         // in [0.70, 1.42): exponent -1 or 0
+    const unsigned bits = __float_as_uint(p);
+    const unsigned long long sig = (bits & 0x7FFFFFu) | 0x800000u;     // p = sig * 2^(e - 23)
+    const int sh = (int)(bits >> 23) - 127 + ni + 17;                  // p * 2^(n + 40) = sig * 2^sh, sh in [-48, 17]
+    return sh >= 0 ? sig << sh : sig >> min(-sh, 63);
 }
 
 __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
@@ -41,19 +52,20 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
     return v;
 }
 
-__global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__restrict__ logits, int64_t vocab,
+__global__ void __launch_bounds__(kSampleThreads, 4) sample_kernel(const float *__restrict__ logits, int64_t vocab,
                                                                 const int32_t *__restrict__ parent,
                                                                 const float *__restrict__ uniforms, int T, float c,
-                                                                int32_t *__restrict__ target) {
+                                                                int64_t rows, int32_t *__restrict__ target) {
     pdl_wait();
     pdl_launch_dependents();
     __shared__ float wmax[kSampleThreads / 32];
     __shared__ unsigned long long tile_sum[kSampleMaxTiles];
     __shared__ float u_s;
-    const int64_t row = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const float *src = logits + row * vocab;
     const bool vec = (vocab & 3) == 0;   // rows are then 16-byte aligned (the base pointer is)
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    __syncthreads();   // the shared scratch of the previous row is free
+    const float *src = logits + row * vocab;
 
     if (tid == 0) {   // level of this node: its uniform is shared by all nodes of the level
         const int b = (int)(row / T), j = (int)(row % T);
@@ -73,7 +85,21 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__r
     float m = -INFINITY;
     if (vec) {
         const float4 *v4 = reinterpret_cast<const float4 *>(src);
-        for (int64_t i = tid; i < vocab / 4; i += kSampleThreads) {
+        const int64_t n4 = vocab / 4;
+        int64_t i = tid;
+        for (; i + 3 * kSampleThreads < n4; i += 4 * kSampleThreads) {   // four loads in flight per thread
+            float4 a[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) a[q] = v4[i + q * kSampleThreads];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (a[q].x > m) m = a[q].x;
+                if (a[q].y > m) m = a[q].y;
+                if (a[q].z > m) m = a[q].z;
+                if (a[q].w > m) m = a[q].w;
+            }
+        }
+        for (; i < n4; i += kSampleThreads) {
             const float4 a = v4[i];
             if (a.x > m) m = a.x;
             if (a.y > m) m = a.y;
@@ -91,9 +117,9 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__r
     __syncthreads();
     m = wmax[0];
     for (int k = 1; k < kSampleThreads / 32; ++k) m = fmaxf(m, wmax[k]);
-    if (m == -INFINITY) {   // nothing has weight
+    if (m == -INFINITY) {   // nothing has weight (the same m in every thread)
         if (tid == 0) target[row] = 0;
-        return;
+        continue;
     }
 
     // ---- integer weights, summed per tile of kSampleTile logits (a warp per tile)
@@ -102,11 +128,18 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__r
         const int64_t base = (int64_t)t * kSampleTile;
         unsigned long long s = 0;
         if (vec) {
-            for (int k = lane * 4; k < kSampleTile; k += 128) {
-                if (base + k < vocab) {
-                    const float4 a = *reinterpret_cast<const float4 *>(src + base + k);
-                    s += sample_weight(a.x, m, c) + sample_weight(a.y, m, c) + sample_weight(a.z, m, c) + sample_weight(a.w, m, c);
+#pragma unroll
+            for (int k0 = 0; k0 < kSampleTile; k0 += 8 * 128) {   // eight loads in flight per lane
+                float4 a[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int k = k0 + q * 128 + lane * 4;
+                    a[q] = base + k < vocab ? __ldcs(reinterpret_cast<const float4 *>(src + base + k))   // last use of the row
+                                            : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);  // weight 0
                 }
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    s += sample_weight(a[q].x, m, c) + sample_weight(a[q].y, m, c) + sample_weight(a[q].z, m, c) + sample_weight(a[q].w, m, c);
             }
         } else {
             for (int k = lane; k < kSampleTile; k += 32)
@@ -118,13 +151,13 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__r
     __syncthreads();
 
     // ---- threshold, crossing tile, crossing element (warp 0)
-    if (warp != 0) return;
+    if (warp != 0) continue;
     unsigned long long total = 0;
     for (int t = lane; t < n_tiles; t += 32) total += tile_sum[t];
     total = warp_sum(total);
     if (total == 0) {
         if (lane == 0) target[row] = 0;
-        return;
+        continue;
     }
     const unsigned long long U = __float2ull_rz(__fmul_rn(u_s, 16777216.0f));
     const unsigned long long thr = (__umul64hi(total, U) << 40) | ((total * U) >> 24);
@@ -170,12 +203,14 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const float *__r
         }
         target[row] = (int32_t)v;
     }
+  }
 }
 
 void launch_sample(const float *logits, int64_t rows, int64_t vocab, const int32_t *parent, const float *uniforms,
-                   int T, float c, int32_t *target, cudaStream_t st) {
+                   int T, float c, int32_t *target, int n_sm, cudaStream_t st) {
     if (rows <= 0) return;
-    launch_pdl(sample_kernel, dim3((unsigned)rows), dim3(kSampleThreads), 0, st, logits, vocab, parent, uniforms, T, c, target);
+    const int64_t ctas = rows < 8 * (int64_t)n_sm ? rows : 8 * (int64_t)n_sm;
+    launch_pdl(sample_kernel, dim3((unsigned)ctas), dim3(kSampleThreads), 0, st, logits, vocab, parent, uniforms, T, c, rows, target);
 }
 
 int sample_max_vocab() { return kSampleTile * kSampleMaxTiles; }
