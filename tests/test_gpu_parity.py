@@ -394,6 +394,50 @@ def test_whole_step_then_next_step_sees_committed_rows(rd):
     assert np.abs(got1 - got2).max() > 1e-3      # the second step really attended to more keys
 
 
+def test_no_call_writes_outside_its_buffers(rd):
+    """Every output and the workspace sit between guard bands filled with a pattern; after a whole
+    step (attention with several M tiles and split units, acceptance, commit) the bands are intact."""
+    from paper_2508_09072_b200 import binding
+    GUARD = 4096
+
+    def guarded(shape, dtype):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        n_al = (n + 255) // 256 * 256
+        raw = torch.full((GUARD + n_al + GUARD,), 0xA5, dtype=torch.uint8, device="cuda")
+        return raw, raw[GUARD:GUARD + n].view(dtype).view(shape)
+
+    def intact(raw, n_bytes):
+        n_al = (n_bytes + 255) // 256 * 256
+        return bool((raw[:GUARD] == 0xA5).all()) and bool((raw[GUARD + n_al:] == 0xA5).all())
+
+    w = W.build_workload("g", 4711, [333, 70, 0, 129], 100, 16, 2, 128, lambda r: W.capped_recursive_tree(r, 100, 12, 4),
+                         max_path=12, vocab=1000, shuffle_pages=True, spare_pages=1)
+    d = binding.to_device(w)
+    B, T, Hq, D = d.q.shape
+    bufs = {}
+    for name, shape, dt in [("out", (B, T, Hq, D), torch.bfloat16), ("lse", (B, T, Hq), torch.float32),
+                            ("status", (B,), torch.int32), ("tgt", (B, T), torch.int32),
+                            ("path", (B, w.max_path), torch.int32), ("n_acc", (B,), torch.int32),
+                            ("bonus", (B,), torch.int32), ("astat", (B,), torch.int32),
+                            ("slots", (B, w.max_path), torch.int32), ("cstat", (B,), torch.int32)]:
+        bufs[name] = guarded(shape, dt)
+    need = rd.workspace_bytes(B, T, Hq, w.n_kv_heads, D)
+    ws_raw, ws = guarded((need,), torch.uint8)
+    t = {k: v[1] for k, v in bufs.items()}
+    rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=t["out"], lse=t["lse"], status=t["status"],
+                   workspace=ws)
+    rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=t["tgt"], workspace=ws,
+              outs=(t["path"], t["n_acc"], t["bonus"], t["astat"]))
+    rd.kv_commit(d.cache, d.k_tree, d.v_tree, t["path"], t["n_acc"], slots=t["slots"], status=t["cstat"])
+    torch.cuda.synchronize()
+    for name, (raw, view) in bufs.items():
+        assert intact(raw, view.numel() * view.element_size()), name
+    assert intact(ws_raw, need), "workspace"
+    assert int(t["status"].max()) == 0 and int(t["astat"].max()) == 0 and int(t["cstat"].max()) == 0
+    got = W.bf16_bits_to_f32(binding.bf16_bits(t["out"])).astype(np.float64)
+    check_attn(w, got, t["status"].cpu().numpy(), t["lse"].cpu().numpy().astype(np.float64))
+
+
 def test_host_side_argument_errors(rd):
     from paper_2508_09072_b200 import binding
     w = W.make("c1", with_logits=False)
