@@ -210,7 +210,7 @@ def test_attn_shared_prefix_equals_duplicated_prefix(rd):
 
 @pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
 def test_attn_full_size_sampled_against_oracle(rd, name):
-    """BASELINE sizes in the launch configuration the benchmark times; the oracle recomputes
+    """Full workload sizes in the launch configuration the benchmark times; the oracle recomputes
     sampled (sequence, KV head) slices one by one."""
     w = W.make(name, with_logits=False)
     got, status, lse = gpu_attn(rd, w)
