@@ -254,7 +254,7 @@ def test_accept_named_workloads_small(rd, name):
     assert np.all(ref["n_acc"] >= w.planted_len)
 
 
-@pytest.mark.parametrize("name", ["c2", "c3"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4"])
 def test_accept_full_size(rd, name):
     w = W.make(name)
     check_accept(w, gpu_accept(rd, w))
@@ -340,6 +340,16 @@ def test_commit_named_workloads_small(rd, name):
         ref = check_commit(w, a["path"], a["n_acc"], update)
         for k in ("k_pool", "v_pool", "seq_lens", "slots", "status"):
             np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+
+
+def test_commit_full_size_c3(rd):
+    """The batched-serving workload at full size: the whole pool (335 MB) is compared byte for byte."""
+    w = W.make("c3")
+    a = oracle.accept(w.parent, w.node_tokens, oracle.argmax(w.logits), w.max_path)
+    got = gpu_commit(rd, w, a["path"], a["n_acc"])
+    ref = check_commit(w, a["path"], a["n_acc"])
+    for k in ("k_pool", "v_pool", "seq_lens", "slots", "status"):
+        np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
 
 
 def test_commit_page_crossing_capacity_and_prefix_guard(rd):
