@@ -49,6 +49,7 @@ def _load():
                                            p32, c_int, p32, p32, c_int, c_int, c_int, c_double,
                                            pd, c_void_p, c_void_p, c_int64, p32]
         lib.oracle_argmax.argtypes = [pf, c_int64, c_int64, p32]
+        lib.oracle_kv_rearrange.argtypes = [p16, p16, c_int, c_int, c_int, c_int, POINTER(c_uint8), p32]
         lib.oracle_sample_targets.argtypes = [pf, p32, pf, c_int, c_int, c_int64, c_double, p32]
         lib.oracle_accept.argtypes = [p32, p32, p32, c_int, c_int, c_int, p32, p32, p32, p32]
         lib.oracle_kv_commit.argtypes = [p16, p16, c_int, c_int, c_int, c_int, p32, c_int, p32, c_int,
@@ -138,6 +139,19 @@ def argmax(logits) -> np.ndarray:
     out = np.zeros(rows, dtype=np.int32)
     _load().oracle_argmax(_ptr(logits, c_float), rows, V, _ptr(out, c_int32))
     return out.reshape(logits.shape[:-1])
+
+
+def kv_rearrange(k, v, valid):
+    """Algorithm 4 on a padded batch cache k, v [B, Hkv, cap, D] (uint16 bf16 bits) with a validity
+    mask [B, cap]; works on copies.  Returns dict(k, v, valid, lengths)."""
+    k, v = _c(k, np.uint16).copy(), _c(v, np.uint16).copy()
+    valid = _c(valid, np.uint8).copy()
+    B, Hkv, cap, D = k.shape
+    assert v.shape == k.shape and valid.shape == (B, cap)
+    lengths = np.zeros(B, dtype=np.int32)
+    _load().oracle_kv_rearrange(_ptr(k, c_uint16), _ptr(v, c_uint16), B, Hkv, cap, D, _ptr(valid, c_uint8),
+                                _ptr(lengths, c_int32))
+    return {"k": k, "v": v, "valid": valid, "lengths": lengths}
 
 
 def sample_targets(logits, parent, uniforms, temperature: float) -> np.ndarray:

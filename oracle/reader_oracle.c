@@ -17,6 +17,8 @@
  *   oracle_accept           invariants 1-3 and the deterministic theorem:
  *                           compare the base model's greedy choice with the
  *                           drafted tokens, keep the longest consistent prefix.
+ *   oracle_kv_rearrange     Sec. 4.3, Algorithm 4 on the padded batch cache:
+ *                           internal padding removed, entries concatenated.
  *   oracle_sample_targets   Appendix C, randomized decoding: x* = F(P, U_t) with
  *                           coupled uniforms, temperature inverse-CDF sampling.
  *   oracle_kv_commit        Sec. 4.3 and Algorithm 4 (KVCacheRearrange): the
@@ -258,6 +260,41 @@ void oracle_argmax(const float *logits, int64_t rows, int64_t vocab, int32_t *ta
  * lowest e among equals.  bonus = target[e] is the token invariant 3 commits
  * after the last accepted one.  path is padded with -1.
  */
+/*
+ * Sec. 4.3 / Algorithm 4 (KVCacheRearrange) on the paper's own layout: a rectangular batch cache
+ * k, v [B][Hkv][cap][D] in which every sample's row of `cap` positions holds real entries and
+ * internal padding.  valid[b][t] != 0 marks a real entry (a mask, not a test for zero values: a
+ * real row may be all zeros).  Per sample: the real entries are moved to the front in their
+ * order (RemoveInternalZeroPadding + TightConcatenate), the vacated tail is zeroed, the mask
+ * becomes 1...10...0 and lengths[b] is the number of real entries.
+ */
+void oracle_kv_rearrange(uint16_t *k, uint16_t *v, int B, int Hkv, int cap, int D,
+                         uint8_t *valid, int32_t *lengths)
+{
+    for (int b = 0; b < B; ++b) {
+        int n = 0;
+        for (int t = 0; t < cap; ++t) {
+            if (!valid[(size_t)b * cap + t]) continue;
+            for (int h = 0; h < Hkv; ++h) {
+                const size_t src = (((size_t)b * Hkv + h) * cap + t) * D;
+                const size_t dst = (((size_t)b * Hkv + h) * cap + n) * D;
+                if (src != dst) {
+                    memmove(k + dst, k + src, (size_t)D * sizeof(uint16_t));
+                    memmove(v + dst, v + src, (size_t)D * sizeof(uint16_t));
+                }
+            }
+            ++n;
+        }
+        for (int h = 0; h < Hkv; ++h) {
+            const size_t at = (((size_t)b * Hkv + h) * cap + n) * D;
+            memset(k + at, 0, (size_t)(cap - n) * D * sizeof(uint16_t));
+            memset(v + at, 0, (size_t)(cap - n) * D * sizeof(uint16_t));
+        }
+        for (int t = 0; t < cap; ++t) valid[(size_t)b * cap + t] = t < n;
+        lengths[b] = n;
+    }
+}
+
 /*
  * Randomized policy of Appendix C ("Randomized decoding"): x* = F(P_theta(. | prefix), U_t), one
  * uniform U_t per output POSITION, shared by the base run and the verifier.  Every node at tree
