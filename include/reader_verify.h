@@ -202,6 +202,20 @@ reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const vo
                                void *stream);
 
 /*
+ * Sec. 4.3 / Algorithm 4 on the paper's own cache layout (not the paged cache of the calls above):
+ * a rectangular batch cache whose per-sample rows hold real entries and internal padding.
+ *   k, v         bf16 [batch][n_kv_heads][capacity][head_dim], compacted in place
+ *   valid        u8   [batch][capacity]: non-zero marks a real entry (a mask; values are not tested
+ *                for zero); rewritten to 1..10..0
+ *   lengths_out  i32  [batch]: real entries per sample
+ * Per sample the real entries move to the front in order (RemoveInternalZeroPadding +
+ * TightConcatenate) and the vacated tail is zeroed.  head_dim a multiple of 8; k, v 16-byte aligned.
+ */
+reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t batch, int32_t n_kv_heads,
+                                  int32_t capacity, int32_t head_dim, uint8_t *valid, int32_t *lengths_out,
+                                  void *stream);
+
+/*
  * reader_accept with target logits, for callers that cannot provide a workspace.  (The paper has
  * no counterpart: this exists only because of how the library is deployed.)  Think of a serving
  * process that gave all device memory to its own pool at start-up, or a decode loop that may not

@@ -25,7 +25,7 @@ NOALLOC_MAX_ROWS = 4096
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
            "reader_set_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
-           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets")
+           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange")
 
 
 class ReaderError(RuntimeError):
@@ -81,6 +81,9 @@ def load_library() -> ctypes.CDLL:
     lib.reader_accept_noalloc.restype = c_int32
     lib.reader_sample_targets.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_int32, c_void_p, c_float, c_void_p, c_void_p]
     lib.reader_sample_targets.restype = c_int32
+    lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
+                                        c_void_p, c_void_p]
+    lib.reader_kv_rearrange.restype = c_int32
     lib.reader_kv_commit.argtypes = [c_void_p, POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
     lib.reader_kv_commit.restype = c_int32
@@ -281,6 +284,19 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_sample_targets")
         return target_ids
+
+    def kv_rearrange(self, k: torch.Tensor, v: torch.Tensor, valid: torch.Tensor,
+                     lengths: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """reader_kv_rearrange: Algorithm 4 on a padded batch cache k, v [B, Hkv, cap, D] with a validity mask
+        [B, cap] (uint8); compacts in place, rewrites the mask, returns the lengths."""
+        _dev(k, torch.bfloat16, "k"); _dev(v, torch.bfloat16, "v"); _dev(valid, torch.uint8, "valid")
+        B, Hkv, cap, D = k.shape
+        if lengths is None:
+            lengths = torch.empty(B, dtype=torch.int32, device=k.device)
+        st = self.lib.reader_kv_rearrange(self._h, _ptr(k), _ptr(v), B, Hkv, cap, D, _ptr(valid), _ptr(lengths), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_kv_rearrange")
+        return lengths
 
     def kv_commit(self, cache: KvCache, k_tree: torch.Tensor, v_tree: torch.Tensor, path: torch.Tensor,
                   n_acc: torch.Tensor, update_seq_lens: bool = True, slots: Optional[torch.Tensor] = None,

@@ -250,6 +250,20 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
     return launch_status();
 }
 
+reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t batch, int32_t n_kv_heads,
+                                  int32_t capacity, int32_t head_dim, uint8_t *valid, int32_t *lengths_out,
+                                  void *stream) {
+    if (!ctx) return READER_ERR_INVALID_ARG;
+    if (batch == 0) return READER_OK;
+    if (!k || !v || !valid || !lengths_out || batch < 0 || n_kv_heads < 1 || capacity < 1 || !aligned16(k) || !aligned16(v))
+        return READER_ERR_INVALID_ARG;
+    if (head_dim < 8 || head_dim % 8 != 0 || head_dim > 256) return READER_ERR_UNSUPPORTED;   // 64 rows are staged in 48 KB
+    if (reader_status st = check_device(ctx)) return st;
+    launch_kv_rearrange(static_cast<__nv_bfloat16 *>(k), static_cast<__nv_bfloat16 *>(v), batch, n_kv_heads, capacity,
+                        head_dim, valid, lengths_out, (cudaStream_t)stream);
+    return launch_status();
+}
+
 reader_status reader_sample_targets(reader_ctx *ctx, const reader_tree *tree, const float *logits, int32_t vocab,
                                     const float *uniforms, float temperature, int32_t *target_ids, void *stream) {
     if (!ctx || !tree) return READER_ERR_INVALID_ARG;

@@ -211,6 +211,8 @@ void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits,
 void launch_sample(const float *logits, int64_t rows, int64_t vocab, const int32_t *parent, const float *uniforms,
                    int T, float c, int32_t *target, int n_sm, cudaStream_t st);
 int sample_max_vocab();
+void launch_kv_rearrange(__nv_bfloat16 *k, __nv_bfloat16 *v, int B, int Hkv, int cap, int D, uint8_t *valid,
+                         int32_t *lengths, cudaStream_t st);
 void launch_accept(const int32_t *parent, const int32_t *tok, int32_t *target, int B, int T,
                    int max_path, const float *part_val, const int32_t *part_idx, int splits,
                    int32_t *path, int32_t *n_acc, int32_t *bonus, int32_t *status, cudaStream_t st);

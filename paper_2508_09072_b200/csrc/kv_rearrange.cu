@@ -1,0 +1,92 @@
+// KVCacheRearrange (Sec. 4.3, Algorithm 4) on the paper's own cache layout: a rectangular batch
+// cache k, v [B][Hkv][cap][D] whose rows hold real entries and internal padding, told apart by a
+// validity mask [B][cap].  Per sample the real entries are moved to the front in order, the tail is
+// zeroed, the mask becomes 1..10..0 and the number of entries is reported.
+//
+// One block per (sample, KV head, K or V) walks its cap positions in chunks of 64: the chunk's mask
+// bytes are prefix-summed, its real rows are staged in shared memory at their compacted places and
+// then written to positions that never lie beyond the chunk's own end -- everything a write can
+// overwrite has been read already, so the compaction is in place.  A chunk that is already where it
+// belongs is not touched.  A second kernel rewrites the mask once every block is done with it.
+#include "common.cuh"
+
+namespace reader {
+
+constexpr int kChunkRows = 64;
+
+__global__ void __launch_bounds__(256) rearrange_rows_kernel(__nv_bfloat16 *__restrict__ k, __nv_bfloat16 *__restrict__ v,
+                                                             int Hkv, int cap, int D,
+                                                             const uint8_t *__restrict__ valid) {
+    pdl_wait();
+    pdl_launch_dependents();
+    extern __shared__ __align__(16) unsigned char stage[];   // kChunkRows rows of D bf16
+    __shared__ int dest[kChunkRows];                          // compacted place within the chunk, or -1
+    __shared__ unsigned bal_s[2];
+    const int bh = blockIdx.x, b = bh / Hkv;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    __nv_bfloat16 *base = (blockIdx.y == 0 ? k : v) + (size_t)bh * cap * D;
+    const uint8_t *mask = valid + (size_t)b * cap;
+    const int pieces_per_row = D / 8;                         // 16-byte pieces
+    uint4 *stage4 = reinterpret_cast<uint4 *>(stage);
+
+    int done = 0;                                             // entries already in place in front
+    for (int c0 = 0; c0 < cap; c0 += kChunkRows) {
+        const int rows = min(kChunkRows, cap - c0);
+        if (warp < 2) {                                       // 64 mask bytes -> two ballots
+            const int r = warp * 32 + lane;
+            const unsigned bal = __ballot_sync(0xffffffffu, r < rows && mask[c0 + r] != 0);
+            if (lane == 0) bal_s[warp] = bal;
+        }
+        __syncthreads();
+        const int count = __popc(bal_s[0]) + __popc(bal_s[1]);
+        if (warp < 2) {                                       // place of every real row among the chunk's real rows
+            const bool real = (bal_s[warp] >> lane) & 1u;
+            dest[warp * 32 + lane] = real ? (warp ? __popc(bal_s[0]) : 0) + __popc(bal_s[warp] & ((1u << lane) - 1)) : -1;
+        }
+        __syncthreads();
+        const bool in_place = done == c0 && count == rows;    // nothing before it was dropped and nothing in it is
+        if (!in_place && count > 0) {
+            for (int i = tid; i < rows * pieces_per_row; i += blockDim.x) {
+                const int r = i / pieces_per_row, piece = i - r * pieces_per_row;
+                const int d = dest[r];
+                if (d >= 0) stage4[d * pieces_per_row + piece] = reinterpret_cast<const uint4 *>(base + (size_t)(c0 + r) * D)[piece];
+            }
+            __syncthreads();                                   // the whole chunk is read before any of it is overwritten
+            uint4 *out = reinterpret_cast<uint4 *>(base + (size_t)done * D);
+            for (int i = tid; i < count * pieces_per_row; i += blockDim.x) out[i] = stage4[i];
+        }
+        done += count;
+        __syncthreads();                                       // stage, dest and the ballots are reused
+    }
+    // the vacated tail
+    uint4 *tail = reinterpret_cast<uint4 *>(base + (size_t)done * D);
+    for (size_t i = tid; i < (size_t)(cap - done) * pieces_per_row; i += blockDim.x) tail[i] = make_uint4(0, 0, 0, 0);
+}
+
+__global__ void __launch_bounds__(256) rearrange_mask_kernel(uint8_t *__restrict__ valid, int cap,
+                                                             int32_t *__restrict__ lengths) {
+    pdl_wait();
+    pdl_launch_dependents();
+    __shared__ int total;
+    const int b = blockIdx.x;
+    uint8_t *mask = valid + (size_t)b * cap;
+    if (threadIdx.x == 0) total = 0;
+    __syncthreads();
+    int n = 0;
+    for (int t = threadIdx.x; t < cap; t += blockDim.x) n += mask[t] != 0;
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_xor_sync(0xffffffffu, n, d);
+    if ((threadIdx.x & 31) == 0) atomicAdd(&total, n);
+    __syncthreads();
+    n = total;
+    for (int t = threadIdx.x; t < cap; t += blockDim.x) mask[t] = t < n;
+    if (threadIdx.x == 0) lengths[b] = n;
+}
+
+void launch_kv_rearrange(__nv_bfloat16 *k, __nv_bfloat16 *v, int B, int Hkv, int cap, int D, uint8_t *valid,
+                         int32_t *lengths, cudaStream_t st) {
+    if (B <= 0) return;
+    launch_pdl(rearrange_rows_kernel, dim3(B * Hkv, 2), dim3(256), (size_t)kChunkRows * D * 2, st, k, v, Hkv, cap, D, valid);
+    launch_pdl(rearrange_mask_kernel, dim3(B), dim3(256), 0, st, valid, cap, lengths);
+}
+
+}  // namespace reader
