@@ -268,6 +268,7 @@ def run_ours(args):
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
+    stall_suspected = False   # set below if the main loop is far slower than the sum of its calls
     assert int(status.max().item()) == 0 and int(cstat.max().item()) == 0 and int(acc_out[3].max().item()) == 0
 
     # ---- per-call and per-kernel breakdown: a second, shorter loop with events between the calls and,
@@ -278,15 +279,19 @@ def run_ours(args):
     kev = [(mk(), mk()) for _ in range(Kb)]
     for a, b in kev:                                  # create the handles
         a.record(); b.record()
+    worst = torch.zeros((), dtype=torch.int32, device=dev)   # a bounded wait that gave up shows in the status words
     for i in range(Kb):
         rd.set_timing_events(*kev[i])
         step(evs[i])
+        worst = torch.maximum(worst, torch.maximum(status.max(), cstat.max()))
     barrier()
     rd.set_timing_events(None, None)
+    assert int(worst.item()) == 0, f"status {int(worst.item())} seen during the breakdown loop"
     t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / Kb
     t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / Kb
     t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / Kb
     t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
+    stall_suspected = ms_total / K > 3.0 * (t_attn_call + t_accept + t_commit)
 
     # ---- the sampling policy's target kernel (an alternative to the argmax; not part of the step)
     uni = torch.rand((B, T), dtype=torch.float32, device=dev)
@@ -300,6 +305,27 @@ def run_ours(args):
     s1.record()
     barrier()
     t_sample = s0.elapsed_time(s1) / 20
+
+    # ---- the paper's own cache maintenance (Algorithm 4) on a padded batch cache of the same size class
+    # (not part of the step: the paged cache needs no such pass)
+    capR, gen = 4096, torch.Generator(device=dev)
+    gen.manual_seed(1234 + rank)
+    kR = torch.randn((B, w.n_kv_heads, capR, w.head_dim), device=dev, generator=gen).to(torch.bfloat16)
+    vR = kR.clone()
+    maskR0 = (torch.rand((B, capR), device=dev, generator=gen) < 0.85).to(torch.uint8)
+    maskR0[:, : capR // 2] = 1                               # the first half is already compact
+    maskR, lenR = maskR0.clone(), torch.empty(B, dtype=torch.int32, device=dev)
+    rd.kv_rearrange(kR, vR, maskR, lenR)
+    r_times = []
+    for _ in range(5):
+        maskR.copy_(maskR0)                                  # same holes again (the data has moved; the cost is the same)
+        r0, r1 = mk(), mk()
+        r0.record(); rd.kv_rearrange(kR, vR, maskR, lenR); r1.record()
+        torch.cuda.synchronize()
+        r_times.append(r0.elapsed_time(r1))
+    t_rearr = sorted(r_times)[len(r_times) // 2]
+    rearr_bytes = 2 * 2 * (B * w.n_kv_heads * (capR - capR // 2) * w.head_dim * 2)   # K and V, read + write of the moving half
+    del kR, vR
 
     # ---- end to end: host buffers in, results out, every step
     host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits")}
@@ -352,6 +378,9 @@ def run_ours(args):
             "accept": {"call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
                        "gbs": w.logits_bytes() / (t_accept * 1e-3) / 1e9},
             "kv_commit": {"call_ms": t_commit},
+            "kv_rearrange": {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,
+                             "note": "Algorithm 4 on a padded batch cache [B][Hkv][4096][D], 85 % valid behind a compact "
+                                     "first half; not in the step"},
             "sample_targets": {"call_ms": t_sample, "algorithmic_bytes": w.logits_bytes(),
                                "gbs": w.logits_bytes() / (t_sample * 1e-3) / 1e9,
                                "note": "sampling policy (Appendix C); replaces the argmax when used; not in the step"},
@@ -377,7 +406,7 @@ def run_ours(args):
             "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args.workload),
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke},
-            "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "roofline_verify_attn": roof_attn,
+            "stall_suspected": bool(stall_suspected), "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "roofline_verify_attn": roof_attn,
             "kernels": kernels,
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -66,7 +66,7 @@ struct Cfg {
 
 struct Bars {
     uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
-    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full[2], pv_done;
+    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full[2], pv_done[2];
     uint32_t tmem_base;
     int32_t abort;
 };
@@ -218,7 +218,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         }
         mbar_init(bar(&bars->p_full[0]), kTileM);
         mbar_init(bar(&bars->p_full[1]), kTileM);
-        mbar_init(bar(&bars->pv_done), 1);
+        mbar_init(bar(&bars->pv_done[0]), 1);
+        mbar_init(bar(&bars->pv_done[1]), 1);
         bars->abort = 0;
         fence_mbar_init();
         fence_proxy_async();
@@ -385,7 +386,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                                         kIdescPV, (tl | kk) != 0);
                     mma_commit(bar(&bars->v_empty[stage]));
                     mma_commit(bar(&bars->s_empty[i & 1]));
-                    mma_commit(bar(&bars->pv_done));
+                    mma_commit(bar(&bars->pv_done[i & 1]));
                 }
                 __syncwarp();
             }
@@ -482,9 +483,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
 
                 if (raise && !first) {
-                    // O may only be rescaled once the previous value product is complete (the scores of
-                    // this tile exist, so product it-2 is complete and the parity wait is unambiguous)
-                    wait(bar(&bars->pv_done), (it - 1) & 1, abort_s, p.error_flag);
+                    // O may only be rescaled once the previous value product is complete
+                    wait(bar(&bars->pv_done[(it - 1) & 1]), ((it - 1) >> 1) & 1, abort_s, p.error_flag);
                     tc_fence_after();
 #pragma unroll 1
                     for (int c = 0; c < D; c += 32) {
@@ -507,11 +507,15 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             }
 
             // ---- segment epilogue
-            // A parity wait can only tell the barrier's current phase from the one before it.  This
-            // warp may have run a tile ahead, so all it knows is that product it-3 is complete: it
-            // waits for product it-2 first, then for the last one.
-            if (it >= 2) wait(bar(&bars->pv_done), (it - 2) & 1, abort_s, p.error_flag);
-            wait(bar(&bars->pv_done), (it - 1) & 1, abort_s, p.error_flag);
+            // The last value product (products complete in issue order, so the others are done too).
+            // A parity wait can only tell a barrier's current phase from the one before it, which is
+            // why the completions alternate between two barriers: when a thread waits for product i on
+            // barrier i & 1, product i-2 is complete (the scores of tile i existed) and product i+2
+            // cannot have been issued (it needs this thread's P), so the barrier is at most one phase
+            // ahead of the waiter.  With a single barrier a thread arriving here after BOTH of the last
+            // two products had completed saw the parity it was waiting to change and slept until the
+            // watchdog woke it, about once in a thousand calls.
+            wait(bar(&bars->pv_done[(it - 1) & 1]), ((it - 1) >> 1) & 1, abort_s, p.error_flag);
             tc_fence_after();
             if (sg.full) {
                 const float inv = 1.f / l;   // l > 0 on a valid row: every node sees itself

@@ -404,6 +404,29 @@ def test_whole_step_then_next_step_sees_committed_rows(rd):
     assert np.abs(got1 - got2).max() > 1e-3      # the second step really attended to more keys
 
 
+def test_thousands_of_calls_never_hit_a_bounded_wait(rd):
+    """Every device-side wait is bounded, so a lost wake-up shows as READER_ERR_TIMEOUT in the status
+    words of one call in many (and as a one-second stall) rather than as a hang.  The status maximum
+    is accumulated on the device over thousands of back-to-back calls on two workloads."""
+    from paper_2508_09072_b200 import binding
+    for name, n in (("c3", 4000), ("c2", 4000)):
+        w = W.make(name, with_logits=False)
+        d = binding.to_device(w, with_logits=False)
+        out = torch.empty_like(d.q)
+        status = torch.empty(w.batch, dtype=torch.int32, device="cuda")
+        ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+        worst = torch.zeros((), dtype=torch.int32, device="cuda")
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(n):
+            rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=out, status=status, workspace=ws)
+            worst = torch.maximum(worst, status.max())
+        t1.record()
+        torch.cuda.synchronize()
+        assert int(worst) == 0, f"{name}: status {int(worst)} seen in {n} calls"
+        assert t0.elapsed_time(t1) < 0.9 * 1000 + n * 1.0, name      # no one-second stall hidden in the run
+
+
 def test_no_call_writes_outside_its_buffers(rd):
     """Every output and the workspace sit between guard bands filled with a pattern; after a whole
     step (attention with several M tiles and split units, acceptance, commit) the bands are intact."""
