@@ -466,6 +466,60 @@ def run_sweep(args):
     rd.close()
 
 
+# ------------------------------------------------------------------------------------------------
+# verify attention alone on all five workloads (cold L2): the numbers behind the roofline table
+# ------------------------------------------------------------------------------------------------
+def run_attn_table(args):
+    import torch
+    from paper_2508_09072_b200 import binding, workloads as W
+    torch.cuda.set_device(0)
+    rd = binding.Reader(0)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    peaks, peak_kind = load_peaks()
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    rows = []
+    for name in ("c1", "c2", "c3", "c4", "c5"):
+        w = W.make(name, with_logits=False)
+        d = binding.to_device(w, with_logits=False)
+        anc, _, _ = rd.tree_encode(d.parent)
+        out = torch.empty_like(d.q)
+        st = torch.empty(w.batch, dtype=torch.int32, device="cuda")
+        ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+        call = lambda: rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out,
+                                      status=st, workspace=ws)
+        for _ in range(5):
+            call()
+        tk, tc = [], []
+        for _ in range(args.sweep_iters):                     # kernel alone (events inside the call)
+            flush.zero_()
+            c, e = mk(), mk()
+            c.record(); e.record()
+            rd.set_timing_events(c, e)
+            call()
+            torch.cuda.synchronize()
+            tk.append(c.elapsed_time(e))
+        rd.set_timing_events(None, None)
+        for _ in range(args.sweep_iters):                     # whole call, launches overlapping as in production
+            flush.zero_()
+            a, b = mk(), mk()
+            a.record(); call(); b.record()
+            torch.cuda.synchronize()
+            tc.append(a.elapsed_time(b))
+        assert int(st.max().item()) == 0
+        k, c_ = sorted(tk)[len(tk) // 2] * 1e-3, sorted(tc)[len(tc) // 2] * 1e-3
+        by, fl = w.attn_algorithmic_bytes(), w.attn_algorithmic_flops()
+        t_hbm, t_tc = by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops_sustained"] * 1e12)
+        rows.append({"workload": name, "kernel_us": k * 1e6, "call_us": c_ * 1e6, "algorithmic_bytes": by,
+                     "algorithmic_flops": fl, "gbs": by / k / 1e9, "hbm_frac": by / k / 1e9 / peaks["hbm_gbs"],
+                     "tflops": fl / k / 1e12, "tensor_frac": fl / k / 1e12 / peaks["bf16_tflops_sustained"],
+                     "binding_bound": "hbm" if t_hbm >= t_tc else "tensor", "binding_frac": max(t_hbm, t_tc) / k,
+                     "tokens_per_s_call": w.batch * w.n_nodes / c_})
+        del d, out
+    print(json.dumps({"table": "verify attention per workload, L2 flushed before every call, median", "peaks": peaks,
+                      "peak_kind": peak_kind, "rows": rows}))
+    rd.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -478,8 +532,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-tree", action="store_true", help="measure the attention call for several tree sizes instead")
     ap.add_argument("--sweep-iters", type=int, default=15)
+    ap.add_argument("--attn-table", action="store_true", help="verify attention alone on C1..C5 instead")
     args = ap.parse_args()
-    if args.sweep_tree:
+    if args.attn_table:
+        run_attn_table(args)
+    elif args.sweep_tree:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
