@@ -293,6 +293,31 @@ def run_ours(args):
     t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
     stall_suspected = ms_total / K > 3.0 * (t_attn_call + t_accept + t_commit)
 
+    # ---- the same step captured once in a CUDA graph and replayed (no host work per step)
+    t_graph = None
+    try:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+        torch.cuda.synchronize()
+        for _ in range(5):
+            graph.replay()
+        Kg = max(3, min(K, 500))
+        barrier()
+        g0, g1 = mk(), mk()
+        g0.record()
+        for _ in range(Kg):
+            graph.replay()
+        g1.record()
+        barrier()
+        t_graph = g0.elapsed_time(g1) / Kg
+    except Exception as exc:                                  # reported, never hidden
+        t_graph = f"capture failed: {exc}"
+
     # ---- the sampling policy's target kernel (an alternative to the argmax; not part of the step)
     uni = torch.rand((B, T), dtype=torch.float32, device=dev)
     tgt_s = torch.empty((B, T), dtype=torch.int32, device=dev)
@@ -406,7 +431,7 @@ def run_ours(args):
             "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args.workload),
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke},
-            "stall_suspected": bool(stall_suspected), "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "roofline_verify_attn": roof_attn,
+            "cuda_graph_replay": ({"ms_per_step": t_graph, "value": B * T * world / (t_graph * 1e-3)} if isinstance(t_graph, float) else t_graph), "stall_suspected": bool(stall_suspected), "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "roofline_verify_attn": roof_attn,
             "kernels": kernels,
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -404,6 +404,49 @@ def test_whole_step_then_next_step_sees_committed_rows(rd):
     assert np.abs(got1 - got2).max() > 1e-3      # the second step really attended to more keys
 
 
+def test_whole_step_captured_in_a_cuda_graph_replays_identically(rd):
+    """A decode step makes no host round trip, so it can be captured once and replayed (what a
+    multi-layer model does per layer): the replay must leave exactly what the eager calls leave."""
+    from paper_2508_09072_b200 import binding
+    w = W.make("c3", reduced=True)
+    d = binding.to_device(w)
+    B, T = w.batch, w.n_nodes
+    out = torch.empty_like(d.q)
+    status = torch.empty(B, dtype=torch.int32, device="cuda")
+    ws = rd.workspace(B, T, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    tgt = torch.empty((B, T), dtype=torch.int32, device="cuda")
+    outs = tuple(torch.empty(sh, dtype=torch.int32, device="cuda") for sh in ((B, w.max_path), (B,), (B,), (B,)))
+    slots = torch.empty((B, w.max_path), dtype=torch.int32, device="cuda")
+    cst = torch.empty(B, dtype=torch.int32, device="cuda")
+    seq0 = d.cache.seq_lens.clone()
+
+    def step():
+        d.cache.seq_lens.copy_(seq0)
+        rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=out, status=status, workspace=ws)
+        rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=tgt, workspace=ws, outs=outs)
+        rd.kv_commit(d.cache, d.k_tree, d.v_tree, outs[0], outs[1], slots=slots, status=cst)
+
+    step()
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (out, tgt, outs[0], outs[1], outs[2], slots, d.cache.k_pool, d.cache.v_pool, d.cache.seq_lens)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()                                   # first use on this stream happens outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for t in (out, tgt, outs[0], outs[1], outs[2], slots):
+        t.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (out, tgt, outs[0], outs[1], outs[2], slots, d.cache.k_pool, d.cache.v_pool, d.cache.seq_lens)):
+        assert torch.equal(a, b)
+    assert int(status.max()) == 0 and int(cst.max()) == 0
+
+
 def test_thousands_of_calls_never_hit_a_bounded_wait(rd):
     """Every device-side wait is bounded, so a lost wake-up shows as READER_ERR_TIMEOUT in the status
     words of one call in many (and as a one-second stall) rather than as a hang.  The status maximum
