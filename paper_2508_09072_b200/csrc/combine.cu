@@ -4,16 +4,17 @@
 // kernel are left alone.
 //
 // The work is found without searching: the attention CTA that started a cut unit left a descriptor
-// (unit, last CTA) in the workspace, so block c reads descriptor c and merges the unit's 128
-// rows, 8 per warp in batches of 2 with the loads of a batch all in flight together.  If the
+// (unit, last CTA) in the workspace, so the four blocks (c, 0..3) read descriptor c and merge 32
+// of the unit's 128 rows each, two per warp with their loads in flight together.  If the
 // attention kernel raised the error flag (a bounded wait gave up), no row of the call can be
 // trusted: everything is zeroed and every status word gets the code.
 #include "common.cuh"
 
 namespace reader {
 
-constexpr int kCombineWarps = 16;                       // one block per attention CTA
-constexpr int kRowsPerWarp = kTileM / kCombineWarps;    // 8 rows, merged in batches of kBatch
+constexpr int kCombineWarps = 16;
+constexpr int kRowGroups = 4;                           // blocks per attention CTA, 32 rows each
+constexpr int kRowsPerWarp = kTileM / (kCombineWarps * kRowGroups);   // 2 rows: one batch
 constexpr int kBatch = 2;
 
 __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const AttnParams p) {
@@ -26,8 +27,8 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
     const int W = p.sched.seq_tile_start[p.B];
 
     if (err != 0) {
-        const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-        const size_t me = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+        const size_t nthreads = (size_t)gridDim.x * gridDim.y * blockDim.x;
+        const size_t me = ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
         uint4 *o = reinterpret_cast<uint4 *>(p.out);
         for (size_t i = me; i < (size_t)p.B * p.T * p.Hq * D / 8; i += nthreads) o[i] = make_uint4(0, 0, 0, 0);
         if (p.lse)
@@ -43,7 +44,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
     const bool all_live = W >= n_lanes;   // with fewer tiles than CTAs some ranges are empty
 
     for (int rb = 0; rb < kRowsPerWarp; rb += kBatch) {
-        const int r0 = warp * kRowsPerWarp + rb;
+        const int r0 = (blockIdx.y * kCombineWarps + warp) * kRowsPerWarp + rb;
         if (r0 >= rows) break;
         float mstar[kBatch], lstar[kBatch];
         float4 acc[kBatch];
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
 void launch_combine(const AttnParams &p, cudaStream_t st) {
     if (p.B <= 0) return;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.sched.n_ctas);
+    cfg.gridDim = dim3(p.sched.n_ctas, kRowGroups);
     cfg.blockDim = dim3(kCombineWarps * 32);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
