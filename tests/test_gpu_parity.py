@@ -160,6 +160,29 @@ def test_attn_random_shapes(rd):
             raise AssertionError(f"case {case}: T={T} G={G} Hkv={Hkv} D={D} lens={lens}: {e}")
 
 
+EXTREMES = [
+    # B, T, G, Hkv, D, max committed length
+    (300, 4, 2, 1, 64, 150),      # more sequences than CTAs
+    (2, 128, 32, 1, 128, 200),    # 32 M tiles per KV stream: 9 lanes
+    (1, 128, 64, 1, 64, 130),     # 64 M tiles: 4 lanes
+    (1, 100, 128, 1, 128, 70),    # 100 M tiles, group = tile height: 2 lanes
+    (3, 65, 16, 2, 128, 64),      # 9 M tiles (last one mostly padding rows), exact page multiple
+]
+
+
+@pytest.mark.parametrize("case", range(len(EXTREMES)))
+def test_attn_scheduler_extremes(rd, case):
+    B, T, G, Hkv, D, Lmax = EXTREMES[case]
+    rng = np.random.default_rng(700 + case)
+    lens = [int(x) for x in rng.integers(0, Lmax + 1, size=B)]
+    lens[0] = Lmax
+    w = W.build_workload("x", 7000 + case, lens, T, G * Hkv, Hkv, D,
+                         lambda r: W.capped_recursive_tree(r, T, 12, 4), max_path=12, vocab=16,
+                         shuffle_pages=True, with_logits=False)
+    got, status, lse = gpu_attn(rd, w, kernel=0)
+    check_attn(w, got, status, lse)
+
+
 def test_attn_empty_batch_is_a_no_op(rd):
     from paper_2508_09072_b200 import binding
     w = W.make("c1", with_logits=False)
