@@ -462,25 +462,27 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                     l *= alpha;
                 }
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                float ls[4] = {0.f, 0.f, 0.f, 0.f};
+                // packed fp32x2 arithmetic: one instruction scales two scores, one adds two probabilities
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+                float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 uint32_t pk[32];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float a = ex2(fmaf(__uint_as_float(s0[2 * i]), p.scale_log2, neg_m));
-                    const float b = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), p.scale_log2, neg_m));
-                    ls[i & 3] += a + b;
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s0[2 * i]), __uint_as_float(s0[2 * i + 1])), sc2, nm2);
+                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                    ls2[i & 1] = __fadd2_rn(ls2[i & 1], e);
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
                     pk[i] = *reinterpret_cast<uint32_t *>(&h2);
                 }
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float a = ex2(fmaf(__uint_as_float(s1[2 * i]), p.scale_log2, neg_m));
-                    const float b = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), p.scale_log2, neg_m));
-                    ls[i & 3] += a + b;
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s1[2 * i]), __uint_as_float(s1[2 * i + 1])), sc2, nm2);
+                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                    ls2[i & 1] = __fadd2_rn(ls2[i & 1], e);
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
                     pk[16 + i] = *reinterpret_cast<uint32_t *>(&h2);
                 }
-                l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+                l += (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
 
                 if (raise && !first) {
                     // O may only be rescaled once the previous value product is complete
