@@ -312,6 +312,9 @@ void oracle_kv_rearrange(uint16_t *k, uint16_t *v, int B, int Hkv, int cap, int 
  *   W_v  = trunc(p * 2^(n + 40))                          integer weight, at most 2^40
  *   S    = sum_v W_v (exact, 64-bit);  U = trunc(u * 2^24);  thr = (S * U) >> 24 (exact, 128-bit)
  *   x*   = the first v whose inclusive prefix sum of W exceeds thr      (0 if S = 0)
+ * Top-k filtering (top_k >= 1; 0 = off): tau = the top_k-th largest logit of the row (NaN counts as
+ * -inf); only logits >= tau keep their weight, so logits equal to tau are all kept (the usual
+ * "mask what is below the k-th value" rule) and the kept set can exceed top_k on ties.
  * Ties on "measure-zero boundaries" are thus resolved towards the lower token id.
  */
 static uint64_t sample_weight(float l, float m, float c)
@@ -329,7 +332,13 @@ static uint64_t sample_weight(float l, float m, float c)
     return (uint64_t)ldexpf(p, (int)n + 40);      /* exact scaling, then truncation */
 }
 
-int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double temperature)
+static int cmp_float_desc(const void *a, const void *b)
+{
+    const float x = *(const float *)a, y = *(const float *)b;
+    return (x < y) - (x > y);
+}
+
+int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double temperature, int64_t top_k)
 {
     const float c = (float)(1.4426950408889634 / temperature);
     float m = row[0];
@@ -337,8 +346,16 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
     for (int64_t v = 1; v < vocab; ++v)
         if (row[v] > m) m = row[v];
     if (m == -INFINITY) return 0;                 /* nothing has weight */
+    float tau = -INFINITY;                        /* the top_k-th largest logit */
+    if (top_k > 0 && top_k < vocab) {
+        float *tmp = (float *)malloc((size_t)vocab * sizeof(float));
+        for (int64_t v = 0; v < vocab; ++v) tmp[v] = isnan(row[v]) ? -INFINITY : row[v];
+        qsort(tmp, (size_t)vocab, sizeof(float), cmp_float_desc);
+        tau = tmp[top_k - 1];
+        free(tmp);
+    }
     uint64_t total = 0;
-    for (int64_t v = 0; v < vocab; ++v) total += sample_weight(row[v], m, c);
+    for (int64_t v = 0; v < vocab; ++v) total += row[v] >= tau ? sample_weight(row[v], m, c) : 0;
     if (total == 0) return 0;
     if (!(u >= 0.0f)) u = 0.0f;                              /* u is meant to lie in [0, 1) */
     if (u > 0.99999994f) u = 0.99999994f;
@@ -346,7 +363,7 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
     const uint64_t thr = (uint64_t)(((unsigned __int128)total * U) >> 24);
     uint64_t run = 0;
     for (int64_t v = 0; v < vocab; ++v) {
-        run += sample_weight(row[v], m, c);
+        run += row[v] >= tau ? sample_weight(row[v], m, c) : 0;
         if (run > thr) return (int32_t)v;
     }
     return (int32_t)(vocab - 1);                  /* not reached: thr < total */
@@ -354,7 +371,7 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
 
 /* target[b][j] for every node; uniforms f32 [B][T], entry lv - 1 serves the nodes of level lv. */
 void oracle_sample_targets(const float *logits, const int32_t *parent, const float *uniforms,
-                           int B, int T, int64_t vocab, double temperature, int32_t *target)
+                           int B, int T, int64_t vocab, double temperature, int64_t top_k, int32_t *target)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < (int64_t)B * T; ++r) {
@@ -365,7 +382,7 @@ void oracle_sample_targets(const float *logits, const int32_t *parent, const flo
             const int up = parent[(size_t)b * T + i];
             i = up < i ? up : -1;                 /* a malformed array cannot send the walk astray */
         }
-        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature);
+        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature, top_k);
     }
 }
 

@@ -11,9 +11,9 @@ import oracle
 from paper_2508_09072_b200 import workloads as W
 
 
-def one_row(logits, u, temperature=1.0):
+def one_row(logits, u, temperature=1.0, top_k=0):
     lg = np.asarray(logits, np.float32).reshape(1, 1, -1)
-    return int(oracle.sample_targets(lg, np.array([[-1]], np.int32), np.array([[u]], np.float32), temperature)[0, 0])
+    return int(oracle.sample_targets(lg, np.array([[-1]], np.int32), np.array([[u]], np.float32), temperature, top_k)[0, 0])
 
 
 def test_equal_logits_give_the_floor_of_u_times_vocab():
@@ -47,6 +47,28 @@ def test_low_temperature_is_greedy_and_u_zero_picks_the_first_token_with_weight(
     assert one_row(lg2, 0.0) == 3                      # -inf, NaN and a weight below 2^-64 are never drawn
     assert one_row(np.array([np.nan, np.nan], np.float32), 0.5) == 0
     assert one_row(np.array([-np.inf, -np.inf], np.float32), 0.5) == 0
+
+
+def test_top_k_filtering():
+    rng = np.random.default_rng(8)
+    lg = rng.standard_normal(30).astype(np.float32) * 2
+    order = np.argsort(-lg, kind="stable")
+    for u in (0.0, 0.4, 0.97):
+        assert one_row(lg, u, top_k=1) == int(np.argmax(lg))            # k = 1 is greedy, whatever u
+        assert one_row(lg, u, top_k=30) == one_row(lg, u)               # k = V (and beyond) filters nothing
+        assert one_row(lg, u, top_k=1000) == one_row(lg, u)
+    # frequencies over a grid of uniforms: the softmax restricted to the k best and renormalised
+    k, n = 5, 1 << 13
+    got = np.bincount([one_row(lg, (i + 0.5) / n, 0.9, top_k=k) for i in range(n)], minlength=30) / n
+    z = lg.astype(np.float64) / 0.9
+    p = np.where(np.isin(np.arange(30), order[:k]), np.exp(z - z.max()), 0.0); p /= p.sum()
+    assert np.abs(got - p).max() <= 1.0 / n + 2e-5
+    # ties at the k-th value are all kept: values 5 4 4 4 1 with k = 2 keep the 5 and all three 4s
+    tie = np.array([4.0, 5.0, 4.0, 1.0, 4.0], np.float32)
+    seen = {one_row(tie, (i + 0.5) / 64, top_k=2) for i in range(64)}
+    assert seen == {0, 1, 2, 4}
+    # NaN is never among the k best
+    assert one_row(np.array([np.nan, 1.0, 2.0], np.float32), 0.0, top_k=2) == 1
 
 
 def test_one_uniform_per_tree_level():
