@@ -18,9 +18,9 @@ def rd():
     r.close()
 
 
-def gpu_sample(rd, parent, logits, uniforms, temperature):
+def gpu_sample(rd, parent, logits, uniforms, temperature, top_k=0):
     t = rd.sample_targets(torch.from_numpy(parent).cuda(), torch.from_numpy(logits).cuda(),
-                          torch.from_numpy(uniforms).cuda(), temperature)
+                          torch.from_numpy(uniforms).cuda(), temperature, top_k=top_k)
     torch.cuda.synchronize()
     return t.cpu().numpy()
 
@@ -45,6 +45,37 @@ def test_sample_targets_match_the_oracle(rd, vocab, temperature):
     got = gpu_sample(rd, parent, logits, u, temperature)
     ref = oracle.sample_targets(logits, parent, u, temperature)
     np.testing.assert_array_equal(got, ref)
+
+
+@pytest.mark.parametrize("vocab", [2, 7, 64, 1000, 2049, 4099, 50024])
+@pytest.mark.parametrize("top_k", [1, 2, 5, 50, 1000])
+def test_sample_targets_with_top_k_match_the_oracle(rd, vocab, top_k):
+    rng = np.random.default_rng(vocab * 13 + top_k)
+    B, T = 2, 19
+    parent = np.stack([W.capped_recursive_tree(rng, T, 7, 3), W.star_tree(T)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, vocab)) * 3).astype(np.float32)
+    u = rng.random((B, T)).astype(np.float32)
+    if vocab >= 7:
+        logits[0, 1, :] = rng.integers(0, 3, size=vocab).astype(np.float32)     # massive ties at the k-th value
+        logits[0, 2, :] = 1.5                                                   # all equal: everything is kept
+        logits[0, 3, 3] = np.nan
+        logits[0, 4, :] = np.nan
+        logits[0, 5, : vocab - 1] = -np.inf                                     # fewer finite logits than k
+        logits[1, 2, :] = -rng.random(vocab).astype(np.float32)                 # all negative
+        logits[1, 3, 0], logits[1, 3, 1] = 0.0, -0.0                            # signed zeros compare equal
+    got = gpu_sample(rd, parent, logits, u, 0.8, top_k)
+    ref = oracle.sample_targets(logits, parent, u, 0.8, top_k)
+    np.testing.assert_array_equal(got, ref)
+
+
+def test_sample_targets_top_k_full_vocabulary(rd):
+    rng = np.random.default_rng(6)
+    B, T, V = 2, 16, 128256
+    parent = np.stack([W.capped_recursive_tree(rng, T, 6, 4) for _ in range(B)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, V)) * 2).astype(np.float32)
+    u = rng.random((B, T)).astype(np.float32)
+    for k in (1, 40, 5000):
+        np.testing.assert_array_equal(gpu_sample(rd, parent, logits, u, 0.9, k), oracle.sample_targets(logits, parent, u, 0.9, k))
 
 
 def test_sample_targets_full_vocabulary_and_out_of_range_uniforms(rd):
