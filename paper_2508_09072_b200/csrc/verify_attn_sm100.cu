@@ -1,15 +1,17 @@
 // Tree-masked verify attention (Sec. 3.2) on the sm_100a tensor cores.
 //
-// Two persistent CTAs per SM each walk their range of the flattened split-KV tile list.  For every
-// unit (sequence, KV head, 128 query rows) a CTA computes S = Q K^T and O += P V with tcgen05.mma,
-// one KV tile of 64 keys (one cache page, or 64 tree nodes) at a time:
+// Two persistent CTAs per SM each walk their range of the flattened split-KV tile list (the CTAs of
+// one lane walk the same KV stream, one M tile each: see the work partition in common.cuh).  For
+// every unit (sequence, KV head, 128 query rows) a CTA computes S = Q K^T and O += P V with
+// tcgen05.mma, one KV tile of 64 keys (one cache page, or 64 tree nodes) at a time:
 //
-//   warp 4      producer: K tiles and V tiles travel through two separate rings (3 and 2 slots).  Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages
-//               from the pool, tree tiles from the tree tensors.  A K slot is free again as soon
-//               as its score product has run, long before the tile's value product, so key loads
-//               run far ahead.  Bytes beyond a sequence's length or the tree's end can never
-//               reach a product: scores there are replaced by -inf, and the value product skips
-//               16-key slices past the end and zeroes the tail of the last slice in place.
+//   warp 4      producer: K tiles and V tiles travel through two separate rings (3 and 2 slots).
+//               Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages from the
+//               pool (with an L2 evict-first hint when no other CTA will read them again), tree
+//               tiles from the tree tensors, the 128 query rows of the next segment (node j, group
+//               member g -> row j*G+g) by one 4-D box per 64 columns as soon as the previous
+//               segment's last score product is done.  A K slot is free again as soon as its score
+//               product has run, long before the tile's value product, so key loads run far ahead.
 //   warp 5      issues S[i] = Q K[i]^T as soon as K[i] has landed and score buffer i & 1 is free
 //   warp 6      issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Two issuing warps because
 //               one thread can start a tcgen05.mma only every ~120 cycles: with 8 + 4 of them per
@@ -20,13 +22,20 @@
 //               probabilities (bf16 pairs) are written over the scores they came from and are
 //               the value product's A operand straight from tensor memory.
 //               The same threads write O (or an (m, l, O) partial) at the end of a segment.
-// The 128 query rows of a unit (node j, group member g -> row j*G+g) come in by one 4-D TMA box per
-// 64 columns, issued by the producer as soon as the previous segment's last score product is done.
+//
+// Bytes beyond a sequence's length or the tree's end can never reach a product: scores there are
+// replaced by -inf, and the value product skips 16-key slices past the end and zeroes the tail of
+// the last slice in shared memory first.
 //
 // TMEM: columns 0-127 hold two score buffers of 64 columns (fp32; the first 32 columns of a buffer
 // hold P as bf16 pairs once its softmax is done), columns 128.. hold O (head_dim columns, fp32);
-// lane = query row.  Every wait on an mbarrier is bounded: after one second
-// without progress a CTA raises the error flag in the workspace, stops waiting and runs to its end.
+// lane = query row.
+//
+// Barriers: a parity wait can only tell a barrier's current phase from the one before it, so every
+// barrier that warps reach at different times exists once per score buffer; the waiter for tile i on
+// barrier i & 1 knows that tile i-2 is complete and that tile i+2 cannot have been issued.  Every
+// wait is bounded: after one second without progress a CTA raises the error flag in the workspace,
+// stops waiting and runs to its end.
 #include <cuda.h>
 
 #include <new>
