@@ -157,10 +157,10 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     const int n_tree_tiles = (T + kPage - 1) / kPage;
     const int64_t tiles_bound = (int64_t)B * Hkv * n_mtiles * ((int64_t)cache->max_pages_per_seq + n_tree_tiles);
     if (tiles_bound >= (int64_t)1 << 31) return READER_ERR_UNSUPPORTED;
+    if (n_mtiles > max_ctas(ctx)) return READER_ERR_UNSUPPORTED;   // a lane holds one CTA per M tile of a KV stream
     const WsLayout w = ws_layout(ctx, B, T, D);
     if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
     if (reader_status st = check_device(ctx)) return st;
-    if (B == 0) return READER_OK;
 
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     cudaStream_t st = (cudaStream_t)stream;
