@@ -277,20 +277,24 @@ def run_ours(args):
     Kb = max(3, min(K, 300))
     evs = [[mk() for _ in range(4)] for _ in range(Kb)]
     kev = [(mk(), mk()) for _ in range(Kb)]
-    for a, b in kev:                                  # create the handles
+    aev = [(mk(), mk()) for _ in range(Kb)]
+    for a, b in kev + aev:                            # create the handles
         a.record(); b.record()
     worst = torch.zeros((), dtype=torch.int32, device=dev)   # a bounded wait that gave up shows in the status words
     for i in range(Kb):
         rd.set_timing_events(*kev[i])
+        rd.set_accept_timing_events(*aev[i])
         step(evs[i])
         worst = torch.maximum(worst, torch.maximum(status.max(), cstat.max()))
     barrier()
     rd.set_timing_events(None, None)
+    rd.set_accept_timing_events(None, None)
     assert int(worst.item()) == 0, f"status {int(worst.item())} seen during the breakdown loop"
     t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / Kb
     t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / Kb
     t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / Kb
     t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
+    t_argmax_kernel = sum(a.elapsed_time(b) for a, b in aev) / Kb
     stall_suspected = ms_total / K > 3.0 * (t_attn_call + t_accept + t_commit)
 
     # ---- the same step captured once in a CUDA graph and replayed (no host work per step)
@@ -394,8 +398,8 @@ def run_ours(args):
     ms_e2e = f0.elapsed_time(f1)
 
     # ---- max over ranks
-    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel = max_over_ranks(
-        [ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel], dev, world)
+    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel, t_argmax_kernel = max_over_ranks(
+        [ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel, t_argmax_kernel], dev, world)
 
     if rank == 0:
         tokens = B * T * world
@@ -408,8 +412,9 @@ def run_ours(args):
                             "gbs": attn_bytes / (t_attn_kernel * 1e-3) / 1e9,
                             "algorithmic_flops": attn_flops, "tflops": attn_flops / (t_attn_kernel * 1e-3) / 1e12,
                             "tokens_per_s_call": tokens / (t_attn_call * 1e-3)},
-            "accept": {"call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
-                       "gbs": w.logits_bytes() / (t_accept * 1e-3) / 1e9},
+            "accept": {"ms": t_argmax_kernel, "call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
+                       "gbs": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9,
+                       "note": "ms / gbs: the argmax kernel alone; call_ms adds the acceptance walk"},
             "kv_commit": {"call_ms": t_commit},
             "kv_rearrange": {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,
                              "note": "Algorithm 4 on a padded batch cache [B][Hkv][4096][D], 85 % valid behind a compact "
@@ -434,7 +439,7 @@ def run_ours(args):
                          "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"], "traffic": None,
                          "peak_kind": peak_kind + " (sustained)"}
         # the step's dominant kernel; the attention kernel's own roofline is always reported beside it
-        roof = roof_attn if t_attn_kernel >= t_accept else hbm_roof("accept (target argmax)", kernels["accept"]["gbs"])
+        roof = roof_attn if t_attn_kernel >= t_argmax_kernel else hbm_roof("accept (target argmax)", kernels["accept"]["gbs"])
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -111,6 +111,10 @@ reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
  * `stop` right after it (the preparation and combine kernels lie outside).  NULL, NULL turns it off. */
 reader_status reader_set_timing_events(reader_ctx *ctx, void *start, void *stop);
 
+/* The same for reader_accept called with logits: the events bracket the argmax kernel (the acceptance
+ * walk that follows lies outside).  NULL, NULL turns it off. */
+reader_status reader_set_accept_timing_events(reader_ctx *ctx, void *start, void *stop);
+
 /* Bytes of device scratch that reader_verify_attn / reader_accept need for at most `max_batch`
  * sequences of at most `max_nodes` nodes.  Host call, no CUDA work.  Returns 0 on bad arguments. */
 size_t reader_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes,

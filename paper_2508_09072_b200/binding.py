@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(_HERE, "libreader_verify.so")
 NOALLOC_MAX_ROWS = 4096
 
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
-           "reader_set_timing_events",
+           "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
            "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange")
 
@@ -65,6 +65,8 @@ def load_library() -> ctypes.CDLL:
     lib.reader_set_attn_kernel.restype = c_int32
     lib.reader_set_timing_events.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.reader_set_timing_events.restype = c_int32
+    lib.reader_set_accept_timing_events.argtypes = [c_void_p, c_void_p, c_void_p]
+    lib.reader_set_accept_timing_events.restype = c_int32
     lib.reader_workspace_bytes.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32]
     lib.reader_workspace_bytes.restype = c_size_t
     lib.reader_tree_encode.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -169,6 +171,14 @@ class Reader:
         st = self.lib.reader_set_timing_events(self._h, a, b)
         if st != OK:
             raise ReaderError(st, "reader_set_timing_events")
+
+    def set_accept_timing_events(self, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+        """Events that reader_accept (with logits) records around its argmax kernel; None, None turns it off."""
+        a = None if start is None else c_void_p(start.cuda_event)
+        b = None if stop is None else c_void_p(stop.cuda_event)
+        st = self.lib.reader_set_accept_timing_events(self._h, a, b)
+        if st != OK:
+            raise ReaderError(st, "reader_set_accept_timing_events")
 
     def workspace_bytes(self, max_batch: int, max_nodes: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
         return int(self.lib.reader_workspace_bytes(self._h, max_batch, max_nodes, n_q_heads, n_kv_heads, head_dim))

@@ -73,6 +73,7 @@ reader_status reader_create(reader_ctx **out, int device) {
     ctx->n_sm = n_sm;
     ctx->attn_kernel = 0;
     ctx->ev_start = ctx->ev_stop = nullptr;
+    ctx->ev_acc_start = ctx->ev_acc_stop = nullptr;
     reader_status st = sm100_host_init(&ctx->sm100, device);
     if (st != READER_OK) {
         delete ctx;
@@ -114,6 +115,13 @@ reader_status reader_set_timing_events(reader_ctx *ctx, void *start, void *stop)
     if (!ctx || ((start == nullptr) != (stop == nullptr))) return READER_ERR_INVALID_ARG;
     ctx->ev_start = (cudaEvent_t)start;
     ctx->ev_stop = (cudaEvent_t)stop;
+    return READER_OK;
+}
+
+reader_status reader_set_accept_timing_events(reader_ctx *ctx, void *start, void *stop) {
+    if (!ctx || ((start == nullptr) != (stop == nullptr))) return READER_ERR_INVALID_ARG;
+    ctx->ev_acc_start = (cudaEvent_t)start;
+    ctx->ev_acc_stop = (cudaEvent_t)stop;
     return READER_OK;
 }
 
@@ -243,7 +251,9 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
         unsigned char *ws = static_cast<unsigned char *>(workspace);
         pv = reinterpret_cast<float *>(ws + w.amax_val);
         pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);
+        if (ctx->ev_acc_start) cudaEventRecord(ctx->ev_acc_start, st);
         launch_argmax(logits, rows, vocab, splits, pv, pi, st);
+        if (ctx->ev_acc_stop) cudaEventRecord(ctx->ev_acc_stop, st);
     }
     launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, pv, pi, splits, path_out, n_acc_out,
                   bonus_out, status_out, st);
