@@ -50,7 +50,7 @@ def _load():
                                            pd, c_void_p, c_void_p, c_int64, p32]
         lib.oracle_argmax.argtypes = [pf, c_int64, c_int64, p32]
         lib.oracle_kv_rearrange.argtypes = [p16, p16, c_int, c_int, c_int, c_int, POINTER(c_uint8), p32]
-        lib.oracle_sample_targets.argtypes = [pf, p32, pf, c_int, c_int, c_int64, c_double, c_int64, p32]
+        lib.oracle_sample_targets.argtypes = [pf, p32, pf, c_int, c_int, c_int64, c_double, c_int64, c_float, p32]
         lib.oracle_accept.argtypes = [p32, p32, p32, c_int, c_int, c_int, p32, p32, p32, p32]
         lib.oracle_kv_commit.argtypes = [p16, p16, c_int, c_int, c_int, c_int, p32, c_int, p32, c_int,
                                          p16, p16, c_int, c_int, p32, p32, c_int, c_int, p32, p32]
@@ -154,17 +154,18 @@ def kv_rearrange(k, v, valid):
     return {"k": k, "v": v, "valid": valid, "lengths": lengths}
 
 
-def sample_targets(logits, parent, uniforms, temperature: float, top_k: int = 0) -> np.ndarray:
+def sample_targets(logits, parent, uniforms, temperature: float, top_k: int = 0, top_p: float = 1.0) -> np.ndarray:
     """Appendix C, randomized policy: per-node target id x* = F(P, U) by temperature inverse-CDF
     sampling; uniforms f32 [B, T], entry level-1 serves all nodes of that tree level.  top_k > 0 keeps
-    only the logits that are at least the top_k-th largest of their row (ties kept)."""
+    only the logits that are at least the top_k-th largest of their row (ties kept); top_p < 1 then keeps
+    the smallest set of highest logits whose weight reaches that share (ties kept)."""
     logits, parent, uniforms = _c(logits, np.float32), _c(parent, np.int32), _c(uniforms, np.float32)
     B, T = parent.shape
     V = logits.shape[-1]
     assert logits.shape == (B, T, V) and uniforms.shape == (B, T)
     out = np.zeros((B, T), dtype=np.int32)
     _load().oracle_sample_targets(_ptr(logits, c_float), _ptr(parent, c_int32), _ptr(uniforms, c_float), B, T, V,
-                                  float(temperature), int(top_k), _ptr(out, c_int32))
+                                  float(temperature), int(top_k), float(top_p), _ptr(out, c_int32))
     return out
 
 

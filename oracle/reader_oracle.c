@@ -315,6 +315,10 @@ void oracle_kv_rearrange(uint16_t *k, uint16_t *v, int B, int Hkv, int cap, int 
  * Top-k filtering (top_k >= 1; 0 = off): tau = the top_k-th largest logit of the row (NaN counts as
  * -inf); only logits >= tau keep their weight, so logits equal to tau are all kept (the usual
  * "mask what is below the k-th value" rule) and the kept set can exceed top_k on ties.
+ * Top-p filtering (0 < top_p < 1; >= 1 = off), applied to what top-k left: with S0 the sum of the kept
+ * weights and M = max(1, (S0 * trunc(top_p * 2^24)) >> 24), tau_p is the largest logit value t for
+ * which the weights of all kept logits >= t add up to at least M (the smallest nucleus reaching
+ * top_p, with logits equal to the last admitted value all admitted); only logits >= tau_p stay.
  * Ties on "measure-zero boundaries" are thus resolved towards the lower token id.
  */
 static uint64_t sample_weight(float l, float m, float c)
@@ -332,13 +336,21 @@ static uint64_t sample_weight(float l, float m, float c)
     return (uint64_t)ldexpf(p, (int)n + 40);      /* exact scaling, then truncation */
 }
 
+typedef struct { float l; uint64_t w; } logit_weight;
+
+static int cmp_lw_desc(const void *a, const void *b)
+{
+    const float x = ((const logit_weight *)a)->l, y = ((const logit_weight *)b)->l;
+    return (x < y) - (x > y);
+}
+
 static int cmp_float_desc(const void *a, const void *b)
 {
     const float x = *(const float *)a, y = *(const float *)b;
     return (x < y) - (x > y);
 }
 
-int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double temperature, int64_t top_k)
+int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double temperature, int64_t top_k, float top_p)
 {
     const float c = (float)(1.4426950408889634 / temperature);
     float m = row[0];
@@ -357,6 +369,25 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
     uint64_t total = 0;
     for (int64_t v = 0; v < vocab; ++v) total += row[v] >= tau ? sample_weight(row[v], m, c) : 0;
     if (total == 0) return 0;
+    if (top_p < 1.0f) {                           /* the nucleus among what top-k left */
+        if (!(top_p >= 5.9604645e-8f)) top_p = 5.9604645e-8f;      /* 2^-24; also NaN */
+        uint64_t need = (uint64_t)(((unsigned __int128)total * (uint64_t)(top_p * 16777216.0f)) >> 24);
+        if (need == 0) need = 1;
+        logit_weight *lw = (logit_weight *)malloc((size_t)vocab * sizeof(logit_weight));
+        int64_t n = 0;
+        for (int64_t v = 0; v < vocab; ++v)
+            if (row[v] >= tau) { lw[n].l = row[v]; lw[n].w = sample_weight(row[v], m, c); ++n; }
+        qsort(lw, (size_t)n, sizeof(logit_weight), cmp_lw_desc);
+        uint64_t cum = 0;
+        for (int64_t i = 0; i < n;) {             /* one group of equal logits at a time */
+            int64_t j = i;
+            while (j < n && lw[j].l == lw[i].l) cum += lw[j++].w;
+            if (cum >= need) { tau = lw[i].l; break; }
+            i = j;
+        }
+        free(lw);
+        total = cum;                              /* the weights of the logits >= the new tau */
+    }
     if (!(u >= 0.0f)) u = 0.0f;                              /* u is meant to lie in [0, 1) */
     if (u > 0.99999994f) u = 0.99999994f;
     const uint64_t U = (uint64_t)(u * 16777216.0f);          /* 24 bits */
@@ -371,7 +402,8 @@ int32_t oracle_sample_row(const float *row, int64_t vocab, float u, double tempe
 
 /* target[b][j] for every node; uniforms f32 [B][T], entry lv - 1 serves the nodes of level lv. */
 void oracle_sample_targets(const float *logits, const int32_t *parent, const float *uniforms,
-                           int B, int T, int64_t vocab, double temperature, int64_t top_k, int32_t *target)
+                           int B, int T, int64_t vocab, double temperature, int64_t top_k, float top_p,
+                           int32_t *target)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < (int64_t)B * T; ++r) {
@@ -382,7 +414,7 @@ void oracle_sample_targets(const float *logits, const int32_t *parent, const flo
             const int up = parent[(size_t)b * T + i];
             i = up < i ? up : -1;                 /* a malformed array cannot send the walk astray */
         }
-        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature, top_k);
+        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature, top_k, top_p);
     }
 }
 

@@ -11,9 +11,10 @@ import oracle
 from paper_2508_09072_b200 import workloads as W
 
 
-def one_row(logits, u, temperature=1.0, top_k=0):
+def one_row(logits, u, temperature=1.0, top_k=0, top_p=1.0):
     lg = np.asarray(logits, np.float32).reshape(1, 1, -1)
-    return int(oracle.sample_targets(lg, np.array([[-1]], np.int32), np.array([[u]], np.float32), temperature, top_k)[0, 0])
+    return int(oracle.sample_targets(lg, np.array([[-1]], np.int32), np.array([[u]], np.float32), temperature, top_k,
+                                     top_p)[0, 0])
 
 
 def test_equal_logits_give_the_floor_of_u_times_vocab():
@@ -69,6 +70,32 @@ def test_top_k_filtering():
     assert seen == {0, 1, 2, 4}
     # NaN is never among the k best
     assert one_row(np.array([np.nan, 1.0, 2.0], np.float32), 0.0, top_k=2) == 1
+
+
+def test_top_p_filtering():
+    rng = np.random.default_rng(12)
+    lg = (rng.standard_normal(40) * 2).astype(np.float32)
+    for u in (0.0, 0.5, 0.99):
+        assert one_row(lg, u, top_p=1.0) == one_row(lg, u)                       # off
+        assert one_row(lg, u, top_p=1e-6) == int(np.argmax(lg))                  # a vanishing share: the best token only
+    # frequencies over a grid of uniforms: the softmax restricted to the nucleus (numpy sort + cumsum) and renormalised
+    n = 1 << 13
+    for top_p, top_k in ((0.5, 0), (0.9, 0), (0.8, 10)):
+        z = lg.astype(np.float64) / 0.7
+        p = np.exp(z - z.max())
+        if top_k:
+            p[np.argsort(-lg, kind="stable")[top_k:]] = 0.0
+        p /= p.sum()
+        order = np.argsort(-p, kind="stable")
+        cut = int(np.searchsorted(np.cumsum(p[order]), top_p, side="left")) + 1   # smallest prefix reaching top_p
+        keep = np.zeros(40, bool); keep[order[:cut]] = True
+        q = np.where(keep, p, 0.0); q /= q.sum()
+        got = np.bincount([one_row(lg, (i + 0.5) / n, 0.7, top_k, top_p) for i in range(n)], minlength=40) / n
+        assert np.abs(got - q).max() <= 1.0 / n + 3e-5, (top_p, top_k)
+    # equal logits at the nucleus boundary are admitted together: 3 | 2 2 2 | 0 with a share that needs one of the 2s
+    tie = np.array([2.0, 3.0, 2.0, 0.0, 2.0], np.float32)
+    seen = {one_row(tie, (i + 0.5) / 64, top_p=0.6) for i in range(64)}
+    assert seen == {0, 1, 2, 4}
 
 
 def test_one_uniform_per_tree_level():
