@@ -342,6 +342,16 @@ def run_ours(args):
     s3.record()
     barrier()
     t_sample_topk = s2.elapsed_time(s3) / 10
+    t_sample_variants = {}
+    for label, kw in (("top_p_0.9", dict(top_p=0.9)), ("top_k_50_top_p_0.9", dict(top_k=50, top_p=0.9))):
+        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, **kw)
+        v0, v1 = mk(), mk()
+        v0.record()
+        for _ in range(5):
+            rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, **kw)
+        v1.record()
+        barrier()
+        t_sample_variants[label] = v0.elapsed_time(v1) / 5
 
     # ---- the paper's own cache maintenance (Algorithm 4) on a padded batch cache of the same size class
     # (not part of the step: the paged cache needs no such pass)
@@ -422,6 +432,9 @@ def run_ours(args):
             "sample_targets": {"call_ms": t_sample, "algorithmic_bytes": w.logits_bytes(),
                                "gbs": w.logits_bytes() / (t_sample * 1e-3) / 1e9,
                                "note": "sampling policy (Appendix C); replaces the argmax when used; not in the step"},
+            "sample_targets_top_p": {"call_ms": t_sample_variants,
+                                     "note": "flat synthetic logits: the nucleus for 0.9 does not fit the candidate list, "
+                                             "so top-p alone selects on the whole row (the slow path)"},
             "sample_targets_top_k_50": {"call_ms": t_sample_topk, "note": "same with top-k filtering (one more pass over the logits for k <= 256)"},
         }
         t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)

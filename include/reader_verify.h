@@ -182,6 +182,9 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
  *   temperature > 0
  *   top_k       0 = no filtering; k >= 1 keeps only the logits that are at least the k-th largest of
  *               their row (NaN counts as -inf; logits equal to that value are all kept)
+ *   top_p       >= 1 = no filtering; 0 < p < 1 keeps, of what top_k left, the smallest set of highest
+ *               logits whose weight reaches the share p (logits equal to the last admitted one are
+ *               admitted with it)
  *   target_ids  i32 [batch][n_nodes] out
  * The CDF is integer arithmetic (fp32 weights from a fixed fused-multiply-add polynomial for
  * 2^x, truncated to 40 fractional bits; exact 64-bit sums; threshold (S * trunc(u 2^24)) >> 24;
@@ -190,8 +193,8 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
  * vocab <= 2 Mi.  No workspace.
  */
 reader_status reader_sample_targets(reader_ctx *ctx, const reader_tree *tree, const float *logits, int32_t vocab,
-                                    const float *uniforms, float temperature, int32_t top_k, int32_t *target_ids,
-                                    void *stream);
+                                    const float *uniforms, float temperature, int32_t top_k, float top_p,
+                                    int32_t *target_ids, void *stream);
 
 /*
  * Sec. 4.3 / Algorithm 4 in per-step form.  For k < n_acc[b] the K/V rows of node path[b][k]

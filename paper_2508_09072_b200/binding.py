@@ -81,8 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.reader_accept_noalloc.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.reader_accept_noalloc.restype = c_int32
-    lib.reader_sample_targets.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_int32, c_void_p, c_float, c_int32, c_void_p,
-                                          c_void_p]
+    lib.reader_sample_targets.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_int32, c_void_p, c_float, c_int32, c_float,
+                                          c_void_p, c_void_p]
     lib.reader_sample_targets.restype = c_int32
     lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
                                         c_void_p, c_void_p]
@@ -282,7 +282,7 @@ class Reader:
         return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
 
     def sample_targets(self, parent: torch.Tensor, logits: torch.Tensor, uniforms: torch.Tensor, temperature: float,
-                       target_ids: Optional[torch.Tensor] = None, top_k: int = 0) -> torch.Tensor:
+                       target_ids: Optional[torch.Tensor] = None, top_k: int = 0, top_p: float = 1.0) -> torch.Tensor:
         """reader_sample_targets: per-node target ids of the temperature-sampling policy with one coupled
         uniform per tree level (feed the result to accept(target_ids=...))."""
         _dev(parent, torch.int32, "parent"); _dev(logits, torch.float32, "logits"); _dev(uniforms, torch.float32, "uniforms")
@@ -291,7 +291,7 @@ class Reader:
             target_ids = torch.empty((B, T), dtype=torch.int32, device=parent.device)
         tree = _Tree(B, T, parent.data_ptr(), None)
         st = self.lib.reader_sample_targets(self._h, ctypes.byref(tree), _ptr(logits), logits.shape[-1], _ptr(uniforms),
-                                            float(temperature), int(top_k), _ptr(target_ids), _stream())
+                                            float(temperature), int(top_k), float(top_p), _ptr(target_ids), _stream())
         if st != OK:
             raise ReaderError(st, "reader_sample_targets")
         return target_ids

@@ -275,18 +275,18 @@ reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t bat
 }
 
 reader_status reader_sample_targets(reader_ctx *ctx, const reader_tree *tree, const float *logits, int32_t vocab,
-                                    const float *uniforms, float temperature, int32_t top_k, int32_t *target_ids,
-                                    void *stream) {
+                                    const float *uniforms, float temperature, int32_t top_k, float top_p,
+                                    int32_t *target_ids, void *stream) {
     if (!ctx || !tree) return READER_ERR_INVALID_ARG;
     if (tree->batch == 0) return READER_OK;
     if (!tree->parent || !logits || !uniforms || !target_ids || !aligned16(logits)) return READER_ERR_INVALID_ARG;
     const int B = tree->batch, T = tree->n_nodes;
-    if (B < 0 || T < 1 || T > kMaxNodes || vocab < 1 || top_k < 0 || !(temperature > 0.f) || temperature > 3.0e38f)
+    if (B < 0 || T < 1 || T > kMaxNodes || vocab < 1 || top_k < 0 || !(top_p > 0.f) || !(temperature > 0.f) || temperature > 3.0e38f)
         return READER_ERR_INVALID_ARG;
     if (vocab > sample_max_vocab()) return READER_ERR_UNSUPPORTED;
     if (reader_status st = check_device(ctx)) return st;
     const float c = (float)(1.4426950408889634 / (double)temperature);
-    launch_sample(logits, (int64_t)B * T, vocab, tree->parent, uniforms, T, c, top_k, target_ids, ctx->n_sm, (cudaStream_t)stream);
+    launch_sample(logits, (int64_t)B * T, vocab, tree->parent, uniforms, T, c, top_k, top_p, target_ids, ctx->n_sm, (cudaStream_t)stream);
     return launch_status();
 }
 

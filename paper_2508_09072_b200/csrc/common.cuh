@@ -209,7 +209,7 @@ void launch_combine(const AttnParams &p, cudaStream_t st);
 void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits, float *part_val,
                    int32_t *part_idx, cudaStream_t st);
 void launch_sample(const float *logits, int64_t rows, int64_t vocab, const int32_t *parent, const float *uniforms,
-                   int T, float c, int64_t top_k, int32_t *target, int n_sm, cudaStream_t st);
+                   int T, float c, int64_t top_k, float top_p, int32_t *target, int n_sm, cudaStream_t st);
 int sample_max_vocab();
 void launch_kv_rearrange(__nv_bfloat16 *k, __nv_bfloat16 *v, int B, int Hkv, int cap, int D, uint8_t *valid,
                          int32_t *lengths, cudaStream_t st);

@@ -18,9 +18,9 @@ def rd():
     r.close()
 
 
-def gpu_sample(rd, parent, logits, uniforms, temperature, top_k=0):
+def gpu_sample(rd, parent, logits, uniforms, temperature, top_k=0, top_p=1.0):
     t = rd.sample_targets(torch.from_numpy(parent).cuda(), torch.from_numpy(logits).cuda(),
-                          torch.from_numpy(uniforms).cuda(), temperature, top_k=top_k)
+                          torch.from_numpy(uniforms).cuda(), temperature, top_k=top_k, top_p=top_p)
     torch.cuda.synchronize()
     return t.cpu().numpy()
 
@@ -66,6 +66,39 @@ def test_sample_targets_with_top_k_match_the_oracle(rd, vocab, top_k):
     got = gpu_sample(rd, parent, logits, u, 0.8, top_k)
     ref = oracle.sample_targets(logits, parent, u, 0.8, top_k)
     np.testing.assert_array_equal(got, ref)
+
+
+@pytest.mark.parametrize("vocab", [2, 7, 64, 1000, 2049, 4099, 50024])
+@pytest.mark.parametrize("top_p,top_k", [(0.05, 0), (0.5, 0), (0.9, 0), (0.999, 0), (0.7, 5), (0.9, 50), (0.95, 1000), (1e-7, 0)])
+def test_sample_targets_with_top_p_match_the_oracle(rd, vocab, top_p, top_k):
+    rng = np.random.default_rng(vocab * 17 + int(top_p * 1000) + top_k)
+    B, T = 2, 19
+    parent = np.stack([W.capped_recursive_tree(rng, T, 7, 3), W.star_tree(T)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, vocab)) * 3).astype(np.float32)       # peaked rows: the candidate list suffices
+    logits[1] = (rng.standard_normal((T, vocab)) * 0.2).astype(np.float32)     # flat rows: the select runs on the whole row
+    u = rng.random((B, T)).astype(np.float32)
+    if vocab >= 7:
+        logits[0, 1, :] = rng.integers(0, 3, size=vocab).astype(np.float32)     # massive ties at the boundary
+        logits[0, 2, :] = 1.5                                                   # all equal: one group holds everything
+        logits[0, 3, 3] = np.nan
+        logits[0, 4, :] = np.nan
+        logits[0, 5, : vocab - 1] = -np.inf
+        logits[1, 3, 0], logits[1, 3, 1] = 9.0, 9.0                             # two equal dominant logits
+    got = gpu_sample(rd, parent, logits, u, 0.8, top_k, top_p)
+    ref = oracle.sample_targets(logits, parent, u, 0.8, top_k, top_p)
+    np.testing.assert_array_equal(got, ref)
+
+
+def test_sample_targets_top_p_full_vocabulary(rd):
+    rng = np.random.default_rng(16)
+    B, T, V = 2, 16, 128256
+    parent = np.stack([W.capped_recursive_tree(rng, T, 6, 4) for _ in range(B)]).astype(np.int32)
+    logits = (rng.standard_normal((B, T, V)) * 2).astype(np.float32)
+    logits[1] *= 3.0                                                            # one batch entry much more peaked
+    u = rng.random((B, T)).astype(np.float32)
+    for top_p, top_k in ((0.3, 0), (0.9, 0), (0.9, 40)):
+        np.testing.assert_array_equal(gpu_sample(rd, parent, logits, u, 0.9, top_k, top_p),
+                                      oracle.sample_targets(logits, parent, u, 0.9, top_k, top_p))
 
 
 def test_sample_targets_top_k_full_vocabulary(rd):
