@@ -322,6 +322,33 @@ def run_ours(args):
     except Exception as exc:                                  # reported, never hidden
         t_graph = f"capture failed: {exc}"
 
+    # ---- a 32-layer model's commits: layer by layer against one batched launch (pools of one page per
+    # sequence would do for the copy itself; the step's own pool is reused for every layer here)
+    n_layers = 32
+    layer_caches = [d.cache] * n_layers
+    lk, lv = [d.k_tree] * n_layers, [d.v_tree] * n_layers
+
+    def commits_one_by_one():
+        d.cache.seq_lens.copy_(seq_lens0)
+        for i in range(n_layers):
+            rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc_out[0], acc_out[1], update_seq_lens=(i == n_layers - 1),
+                         slots=slots, status=cstat)
+
+    def commits_batched():
+        d.cache.seq_lens.copy_(seq_lens0)
+        rd.kv_commit_layers(layer_caches, lk, lv, acc_out[0], acc_out[1], slots=slots, status=cstat)
+
+    t_layers = {}
+    for label, fn in (("one_by_one", commits_one_by_one), ("batched", commits_batched)):
+        fn()
+        c0, c1 = mk(), mk()
+        c0.record()
+        for _ in range(20):
+            fn()
+        c1.record()
+        barrier()
+        t_layers[label] = c0.elapsed_time(c1) / 20
+
     # ---- the sampling policy's target kernel (an alternative to the argmax; not part of the step)
     uni = torch.rand((B, T), dtype=torch.float32, device=dev)
     tgt_s = torch.empty((B, T), dtype=torch.int32, device=dev)
@@ -426,6 +453,8 @@ def run_ours(args):
                        "gbs": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9,
                        "note": "ms / gbs: the argmax kernel alone; call_ms adds the acceptance walk"},
             "kv_commit": {"call_ms": t_commit},
+            "kv_commit_32_layers": {"call_ms": t_layers, "note": "the accepted rows committed into 32 layers: 32 calls of "
+                                    "reader_kv_commit against one reader_kv_commit_layers; not in the step"},
             "kv_rearrange": {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,
                              "note": "Algorithm 4 on a padded batch cache [B][Hkv][4096][D], 85 % valid behind a compact "
                                      "first half; not in the step"},

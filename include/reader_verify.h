@@ -212,6 +212,21 @@ reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const vo
                                void *stream);
 
 /*
+ * reader_kv_commit for every layer of a model in one launch (the accepted path is the same in all
+ * layers; a 32-layer model would otherwise issue 32 small kernels per step).
+ *   caches     HOST array [n_layers] of reader_kv_cache: each layer's own k_pool / v_pool; all layers
+ *              must share page_table, seq_lens, num_pages, n_kv_heads, head_dim, max_pages_per_seq and
+ *              shared_prefix_len (one block table for the whole model), else READER_ERR_INVALID_ARG
+ *   k_trees, v_trees  HOST arrays [n_layers] of device pointers, bf16 [batch][n_nodes][n_kv_heads][head_dim]
+ * slots_out, status_out and the seq_lens update are those of reader_kv_commit (the check has the
+ * same outcome in every layer).  n_layers >= 1.
+ */
+reader_status reader_kv_commit_layers(reader_ctx *ctx, const reader_kv_cache *caches, const void *const *k_trees,
+                                      const void *const *v_trees, int32_t n_layers, int32_t batch, int32_t n_nodes,
+                                      const int32_t *path, const int32_t *n_acc, int32_t max_path,
+                                      int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out, void *stream);
+
+/*
  * Sec. 4.3 / Algorithm 4 on the paper's own cache layout (not the paged cache of the calls above):
  * a rectangular batch cache whose per-sample rows hold real entries and internal padding.
  *   k, v         bf16 [batch][n_kv_heads][capacity][head_dim], compacted in place

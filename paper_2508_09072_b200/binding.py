@@ -25,7 +25,7 @@ NOALLOC_MAX_ROWS = 4096
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
            "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
-           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange")
+           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers")
 
 
 class ReaderError(RuntimeError):
@@ -84,6 +84,10 @@ def load_library() -> ctypes.CDLL:
     lib.reader_sample_targets.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_int32, c_void_p, c_float, c_int32, c_float,
                                           c_void_p, c_void_p]
     lib.reader_sample_targets.restype = c_int32
+    lib.reader_kv_commit_layers.argtypes = [c_void_p, POINTER(_KvCache), POINTER(c_void_p), POINTER(c_void_p), c_int32,
+                                            c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p,
+                                            c_void_p]
+    lib.reader_kv_commit_layers.restype = c_int32
     lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
                                         c_void_p, c_void_p]
     lib.reader_kv_rearrange.restype = c_int32
@@ -295,6 +299,28 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_sample_targets")
         return target_ids
+
+    def kv_commit_layers(self, caches, k_trees, v_trees, path: torch.Tensor, n_acc: torch.Tensor,
+                         update_seq_lens: bool = True, slots: Optional[torch.Tensor] = None,
+                         status: Optional[torch.Tensor] = None):
+        """reader_kv_commit_layers: the accepted rows of every layer (lists of KvCache sharing page_table and
+        seq_lens, and of tree K / V tensors) committed in one launch."""
+        n = len(caches)
+        for t in list(k_trees) + list(v_trees):
+            _dev(t, torch.bfloat16, "tree K/V")
+        _dev(path, torch.int32, "path"); _dev(n_acc, torch.int32, "n_acc")
+        B, T = k_trees[0].shape[:2]
+        max_path = path.shape[1]
+        slots = slots if slots is not None else torch.empty((B, max_path), dtype=torch.int32, device=path.device)
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=path.device)
+        c_arr = (_KvCache * n)(*[c._c() for c in caches])
+        k_arr = (c_void_p * n)(*[t.data_ptr() for t in k_trees])
+        v_arr = (c_void_p * n)(*[t.data_ptr() for t in v_trees])
+        st = self.lib.reader_kv_commit_layers(self._h, c_arr, k_arr, v_arr, n, B, T, _ptr(path), _ptr(n_acc), max_path,
+                                              int(bool(update_seq_lens)), _ptr(slots), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_kv_commit_layers")
+        return slots, status
 
     def kv_rearrange(self, k: torch.Tensor, v: torch.Tensor, valid: torch.Tensor,
                      lengths: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -1,6 +1,7 @@
 // C-ABI entry points: argument validation, workspace carving and kernel sequencing.
 // Nothing here touches device data from the host or synchronises the stream.
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 #include "ctx.cuh"
@@ -257,6 +258,41 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
     }
     launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, pv, pi, splits, path_out, n_acc_out,
                   bonus_out, status_out, st);
+    return launch_status();
+}
+
+reader_status reader_kv_commit_layers(reader_ctx *ctx, const reader_kv_cache *caches, const void *const *k_trees,
+                                      const void *const *v_trees, int32_t n_layers, int32_t batch, int32_t n_nodes,
+                                      const int32_t *path, const int32_t *n_acc, int32_t max_path,
+                                      int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out, void *stream) {
+    if (!ctx || !caches || n_layers < 1) return READER_ERR_INVALID_ARG;
+    if (batch == 0) return READER_OK;
+    if (!k_trees || !v_trees || !path || !n_acc || !slots_out || !status_out) return READER_ERR_INVALID_ARG;
+    const reader_kv_cache &c0 = caches[0];
+    if (batch < 0 || n_nodes < 1 || n_nodes > kMaxNodes || max_path < 1 || c0.n_kv_heads < 1 || !c0.page_table ||
+        !c0.seq_lens || c0.max_pages_per_seq < 1 || c0.num_pages < 0 || c0.shared_prefix_len < 0 ||
+        c0.shared_prefix_len % kPage != 0)
+        return READER_ERR_INVALID_ARG;
+    if (c0.page_size != kPage || c0.head_dim % 8 != 0 || c0.head_dim < 8) return READER_ERR_UNSUPPORTED;
+    std::vector<CommitLayers> chunks((n_layers + kCommitLayersPerLaunch - 1) / kCommitLayersPerLaunch);
+    for (int l = 0; l < n_layers; ++l) {
+        const reader_kv_cache &c = caches[l];
+        if (c.page_table != c0.page_table || c.seq_lens != c0.seq_lens || c.num_pages != c0.num_pages ||
+            c.n_kv_heads != c0.n_kv_heads || c.head_dim != c0.head_dim || c.page_size != c0.page_size ||
+            c.max_pages_per_seq != c0.max_pages_per_seq || c.shared_prefix_len != c0.shared_prefix_len ||
+            !c.k_pool || !c.v_pool || !k_trees[l] || !v_trees[l] || !aligned16(c.k_pool) || !aligned16(c.v_pool) ||
+            !aligned16(k_trees[l]) || !aligned16(v_trees[l]))
+            return READER_ERR_INVALID_ARG;
+        CommitLayers &ch = chunks[l / kCommitLayersPerLaunch];
+        const int at = l % kCommitLayersPerLaunch;
+        ch.k_pool[at] = static_cast<__nv_bfloat16 *>(c.k_pool);
+        ch.v_pool[at] = static_cast<__nv_bfloat16 *>(c.v_pool);
+        ch.k_tree[at] = static_cast<const __nv_bfloat16 *>(k_trees[l]);
+        ch.v_tree[at] = static_cast<const __nv_bfloat16 *>(v_trees[l]);
+    }
+    if (reader_status st = check_device(ctx)) return st;
+    launch_kv_commit_layers(c0, chunks.data(), n_layers, batch, n_nodes, path, n_acc, max_path, update_seq_lens,
+                            slots_out, status_out, (cudaStream_t)stream);
     return launch_status();
 }
 

@@ -375,6 +375,41 @@ def test_commit_full_size_c3(rd):
         np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
 
 
+@pytest.mark.parametrize("n_layers", [1, 3, 40])
+def test_commit_all_layers_in_one_launch_equals_layer_by_layer(rd, n_layers):
+    """reader_kv_commit_layers against the oracle applied to every layer's pools (and so against
+    n_layers calls of reader_kv_commit): one sequence without room is refused in every layer."""
+    from paper_2508_09072_b200 import binding
+    T = 20
+    w = W.build_workload("ml", 55, [60, 127, 200, 133, 64], T, 8, 4, 64, lambda r: W.capped_recursive_tree(r, T, 8, 3),
+                         max_path=8, vocab=16, shuffle_pages=True, with_logits=False, spare_pages=2)
+    w.page_table[1, 2:] = -1                                  # sequence 1 has no page for positions >= 128
+    rng = np.random.default_rng(n_layers)
+    path = np.tile(np.arange(8, dtype=np.int32), (5, 1))
+    n_acc = np.array([8, 5, 0, 3, 8], np.int32)
+    page_table = torch.from_numpy(w.page_table).cuda()
+    seq_lens = torch.from_numpy(w.seq_lens).cuda()
+    host, caches, k_trees, v_trees = [], [], [], []
+    for _ in range(n_layers):
+        kp = rng.integers(0, 65535, size=w.k_pool.shape).astype(np.uint16)
+        vp = rng.integers(0, 65535, size=w.k_pool.shape).astype(np.uint16)
+        kt = rng.integers(0, 65535, size=w.k_tree.shape).astype(np.uint16)
+        vt = rng.integers(0, 65535, size=w.k_tree.shape).astype(np.uint16)
+        host.append((kp, vp, kt, vt))
+        caches.append(binding.KvCache(binding.bf16_tensor(kp, "cuda"), binding.bf16_tensor(vp, "cuda"), page_table, seq_lens))
+        k_trees.append(binding.bf16_tensor(kt, "cuda")); v_trees.append(binding.bf16_tensor(vt, "cuda"))
+    slots, status = rd.kv_commit_layers(caches, k_trees, v_trees, torch.from_numpy(path).cuda(), torch.from_numpy(n_acc).cuda())
+    torch.cuda.synchronize()
+    for l, (kp, vp, kt, vt) in enumerate(host):
+        ref = oracle.kv_commit(kp, vp, w.page_table, w.seq_lens, 0, kt, vt, path, n_acc)
+        np.testing.assert_array_equal(binding.bf16_bits(caches[l].k_pool), ref["k_pool"], err_msg=f"layer {l} K")
+        np.testing.assert_array_equal(binding.bf16_bits(caches[l].v_pool), ref["v_pool"], err_msg=f"layer {l} V")
+    np.testing.assert_array_equal(slots.cpu().numpy(), ref["slots"])
+    np.testing.assert_array_equal(status.cpu().numpy(), ref["status"])
+    np.testing.assert_array_equal(seq_lens.cpu().numpy(), ref["seq_lens"])
+    assert ref["status"].tolist() == [0, oracle.CAPACITY, 0, 0, 0]
+
+
 def test_commit_page_crossing_capacity_and_prefix_guard(rd):
     T = 20
     w = W.build_workload("s", 31, [60, 127, 200, 128 + 5, 64], T, 8, 4, 64,
