@@ -2,16 +2,19 @@
  * reader_verify.h -- C ABI of the batched tree-verification step of READER-style lossless
  * speculative decoding, implemented as hand-written CUDA for sm_100a (NVIDIA B200).
  *
- * One decoding step of the method (Algorithm 1, lines 15-16 and 18-20) hands a draft tree per
- * sequence to the target model, which scores every node in one pass (Sec. 3.2), keeps the
- * longest root path the model agrees with (Algorithm 5; Appendix C, invariants 1-3) and appends
- * the accepted entries to the KV cache without gaps (Sec. 4.3, Algorithm 4).  This library is
- * the attention, acceptance and cache part of that step:
+ * One decoding step of the method (Algorithm 1: the Verify call and the cache maintenance that
+ * follows it) hands a draft tree per sequence to the target model, which scores every node in one
+ * pass (Sec. 3.2), keeps the longest root path the model agrees with (Algorithm 5; Appendix C,
+ * invariants 1-3) and appends the accepted entries to the KV cache without gaps (Sec. 4.3,
+ * Algorithm 4).  This library is the attention, acceptance and cache part of that step:
  *
  *     reader_tree_encode   parent array  ->  per-node ancestor bitmask           (Sec. 3.2 mask)
  *     reader_verify_attn   tree-masked attention over paged cache + tree K/V     (Sec. 3.2)
  *     reader_accept        target argmax + longest consistent root path          (Algorithm 5)
  *     reader_kv_commit     accepted K/V rows -> cache tail, seq_lens += n_acc    (Algorithm 4)
+ *   and, beside these: reader_sample_targets (the sampling policies of Appendix C in place of the
+ *   argmax), reader_kv_commit_layers (all layers of a model in one launch), reader_kv_rearrange
+ *   (Algorithm 4 on the paper's padded cache layout), reader_accept_noalloc.
  *
  * Conventions common to every call
  *   - Every pointer named below is a DEVICE pointer owned by the caller unless it says "host".
@@ -152,7 +155,7 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
                                  void *stream);
 
 /*
- * Algorithm 5 step 2 with the greedy policy of Appendix C.  If `logits` (f32
+ * Algorithm 5 (the comparison with the base model's choice) with the greedy policy of Appendix C.  If `logits` (f32
  * [batch][n_nodes][vocab]) is given, target_ids[b][j] is first set to the lowest index of the
  * row maximum (a NaN never wins; a NaN in slot 0 counts as -inf); otherwise target_ids is read
  * as given (any policy's per-node choice, e.g. a sampler driven by coupled uniforms).

@@ -170,7 +170,7 @@ def sample_targets(logits, parent, uniforms, temperature: float, top_k: int = 0,
 
 
 def accept(parent, node_tokens, target_ids, max_path: int):
-    """Longest consistent root path (Algorithm 5 step 2) -> dict(path, n_acc, bonus, status)."""
+    """Longest consistent root path (Algorithm 5) -> dict(path, n_acc, bonus, status)."""
     parent, tok, tgt = _c(parent, np.int32), _c(node_tokens, np.int32), _c(target_ids, np.int32)
     B, T = parent.shape
     path = np.zeros((B, max_path), dtype=np.int32)

@@ -13,7 +13,7 @@
  *   oracle_verify_attn      Sec. 3.2: scaled dot-product attention of the
  *                           gamma tree queries against the s cached keys plus
  *                           the gamma tree keys under that mask.
- *   oracle_argmax /         Algorithm 5 (Verify) step 2 and Appendix C,
+ *   oracle_argmax /         Algorithm 5 (Verify) and Appendix C,
  *   oracle_accept           invariants 1-3 and the deterministic theorem:
  *                           compare the base model's greedy choice with the
  *                           drafted tokens, keep the longest consistent prefix.
@@ -253,7 +253,7 @@ void oracle_argmax(const float *logits, int64_t rows, int64_t vocab, int32_t *ta
 }
 
 /*
- * Algorithm 5 step 2 / Appendix C invariant 2, by brute force: every node e
+ * Algorithm 5 (the longest consistent prefix) / Appendix C invariant 2, by brute force: every node e
  * is tried as the end of a root-to-e path; the path is consistent when every
  * non-root node u on it carries the token the base model picks after its
  * parent, tok[u] == target[parent[u]].  The longest consistent path wins,

@@ -1,4 +1,4 @@
-// Acceptance (Algorithm 5 step 2; Appendix C invariants 2-3 with the greedy policy): row argmax
+// Acceptance (Algorithm 5; Appendix C invariants 2-3 with the greedy policy): row argmax
 // of the target logits with a lowest-index tie-break, then the longest root path whose every
 // non-root node carries the token the target model picks after its parent.
 #include <limits.h>
