@@ -18,7 +18,8 @@ constexpr int kMaxNodes = READER_MAX_NODES;
 //
 // A *unit* is (sequence b, KV head h, M tile mt): kTileM query rows (node j, group member g) with
 // row = j * G + g, attending over ntiles(b) KV tiles: the committed pages of b followed by the
-// tree tiles.  The KV streams (b, h), tiles in order, form one flat list of W tiles that is cut
+// tree tiles.  The KV streams (b, h), each kUnitOverhead overhead entries followed by its tiles in
+// order, form one flat list of W entries that is cut
 // into n_lanes contiguous ranges of near-equal length.  A *lane* is n_mtiles CTAs, one per M tile,
 // that walk the same range: CTA c has lane c / n_mtiles and M tile c % n_mtiles.  The CTAs of a
 // lane read the same K/V tiles at the same pace, so all but the first of them find the tile in
@@ -38,11 +39,18 @@ struct Sched {
 
 struct Segment {
     int b, h, mt;
-    int tile_begin, tile_end;  // within the unit
+    int tile_begin, tile_end;  // real tiles within the unit; may be empty (tile_end <= tile_begin)
+    int span;                  // entries of the flat list this segment covers (overhead entries included)
+    int unit_w0;               // flat index of the unit's first entry
     int ntiles, npages;
     bool full;                 // covers the whole unit
     int slot;                  // partial slot when !full
 };
+
+// Starting a unit costs about as much as kUnitOverhead tiles (waiting for Q, the epilogue, a partial):
+// the flat list gives every unit that many extra entries at its start, so a CTA whose range holds
+// more unit starts gets correspondingly fewer real tiles and all CTAs finish together.
+constexpr int kUnitOverhead = 6;
 
 constexpr int kMinTilesPerCta = 8;
 
@@ -73,13 +81,17 @@ __device__ __forceinline__ Segment segment_at(const Sched &s, int B, int cta, in
     g.b = find_seq(s.seq_tile_start, B, w);
     g.ntiles = s.seq_ntiles[g.b];
     g.npages = s.seq_npages[g.b];
+    const int per_unit = g.ntiles + kUnitOverhead;          // entries of one unit: overhead first, then its tiles
     int local = w - s.seq_tile_start[g.b];
-    int unit = local / g.ntiles;
-    g.tile_begin = local - unit * g.ntiles;
+    int unit = local / per_unit;
+    const int pos = local - unit * per_unit;
+    const int pos_end = min(per_unit, pos + (range_end - w));
+    g.span = pos_end - pos;
+    g.unit_w0 = w - pos;
+    g.tile_begin = max(0, pos - kUnitOverhead);
+    g.tile_end = max(0, pos_end - kUnitOverhead);
     g.h = unit;
     g.mt = cta % s.n_mtiles;
-    int left = range_end - w;
-    g.tile_end = min(g.ntiles, g.tile_begin + left);
     g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
     g.slot = 2 * cta + (g.tile_begin == 0 ? 1 : 0);
     return g;
@@ -99,13 +111,17 @@ __device__ __forceinline__ Segment segment_at_warp(const Sched &s, int B, int ct
     g.b = b;
     g.ntiles = s.seq_ntiles[b];
     g.npages = s.seq_npages[b];
+    const int per_unit = g.ntiles + kUnitOverhead;          // entries of one unit: overhead first, then its tiles
     int local = w - s.seq_tile_start[b];
-    int unit = local / g.ntiles;
-    g.tile_begin = local - unit * g.ntiles;
+    int unit = local / per_unit;
+    const int pos = local - unit * per_unit;
+    const int pos_end = min(per_unit, pos + (range_end - w));
+    g.span = pos_end - pos;
+    g.unit_w0 = w - pos;
+    g.tile_begin = max(0, pos - kUnitOverhead);
+    g.tile_end = max(0, pos_end - kUnitOverhead);
     g.h = unit;
     g.mt = cta % s.n_mtiles;
-    int left = range_end - w;
-    g.tile_end = min(g.ntiles, g.tile_begin + left);
     g.full = (g.tile_begin == 0) && (g.tile_end == g.ntiles);
     g.slot = 2 * cta + (g.tile_begin == 0 ? 1 : 0);
     return g;
@@ -142,11 +158,11 @@ struct SplitDesc {
 
 // Called by one thread per segment: if the segment starts its unit without finishing it, note where
 // the unit's partials end so that the combine kernel can find them without any search.
-__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, int n_lanes, const Segment &g, int cta, int w_seg_begin, int W) {
-    if (g.tile_begin != 0 || g.full) return;
+__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, int n_lanes, const Segment &g, int cta, int W) {
+    if (g.tile_begin != 0 || g.full || g.tile_end <= g.tile_begin) return;
     SplitDesc d;
     d.b = g.b; d.h = g.h; d.mt = g.mt;
-    d.c_last = cta_of_tile(w_seg_begin + g.ntiles - 1, n_lanes, W) * s.n_mtiles + g.mt;   // same M tile, last lane
+    d.c_last = cta_of_tile(g.unit_w0 + kUnitOverhead + g.ntiles - 1, n_lanes, W) * s.n_mtiles + g.mt;   // same M tile, last lane
     desc[cta] = d;
 }
 

@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
         if (lane == 0) seq_tile_start[0] = 0;
         for (int base = 0; base < B; base += 32) {
             int b = base + lane;
-            int v = b < B ? seq_ntiles[b] * units_per_seq : 0;
+            int v = b < B && seq_ntiles[b] > 0 ? (seq_ntiles[b] + kUnitOverhead) * units_per_seq : 0;
             int incl = v;
             for (int d = 1; d < 32; d <<= 1) {
                 int t = __shfl_up_sync(0xffffffffu, incl, d);

@@ -24,8 +24,9 @@ __global__ void __launch_bounds__(kTileM) attn_generic_kernel(const AttnParams p
 
     while (w < w_end) {
         const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
-        if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, w, W);
-        w += sg.tile_end - sg.tile_begin;
+        if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
+        w += sg.span;
+        if (sg.tile_end <= sg.tile_begin) continue;   // the range ended among the unit's overhead entries
 
         const int grow = sg.mt * kTileM + tid;           // row within the (b, h) problem
         const bool row_ok = grow < p.T * p.G;

@@ -141,10 +141,13 @@ struct TileCursor {
         cache_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
     }
     __device__ __forceinline__ void next_segment(const AttnParams &p, int cta, int lane) {
-        active = w < w_end;
+        active = false;
+        while (w < w_end) {   // segments without a real tile (a range that ends among overhead entries) are skipped
+            sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            w += sg.span;
+            if (sg.tile_end > sg.tile_begin) { active = true; break; }
+        }
         if (!active) return;
-        sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
-        w += sg.tile_end - sg.tile_begin;
         L = p.seq_lens[sg.b];
         t = sg.tile_begin;
         refill(p, lane);
@@ -274,7 +277,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             bool moved = false;
             if (q_w < w_end && ready(bar(&bars->q_empty), (q_seg & 1) ^ 1)) {
                 const Segment sg = segment_at_warp(p.sched, p.B, cta, q_w, w_end, lane);
-                q_w += sg.tile_end - sg.tile_begin;
+                q_w += sg.span;
+                if (sg.tile_end <= sg.tile_begin) continue;   // no real tile: no query tile
                 if (lane == 0) {
                     const uint32_t full = bar(&bars->q_full);
                     mbar_arrive_expect_tx(full, C::kQBytes);
@@ -330,7 +334,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         while (w < w_end && !*abort_s) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
-            w += n;
+            w += sg.span;
+            if (n <= 0) continue;
             wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
             for (int t = 0; t < n; ++t, ++i) {
                 const int stage = i % kStagesK, buf = i & 1;
@@ -363,7 +368,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         while (w < w_end && !*abort_s) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
-            w += n;
+            w += sg.span;
+            if (n <= 0) continue;
             const int L = p.seq_lens[sg.b];
             for (int tl = 0; tl < n; ++tl, ++i) {
                 const int stage = i % kStagesV;
@@ -408,8 +414,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         if (tid == 0) p.split_desc[cta].b = -1;
         while (w < w_end) {
             const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
-            if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, w, W);
-            w += sg.tile_end - sg.tile_begin;
+            if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
+            w += sg.span;
+            if (sg.tile_end <= sg.tile_begin) continue;
             const int L = p.seq_lens[sg.b];
             const int grow = sg.mt * kTileM + tid;
             const bool row_ok = grow < p.T * p.G;
