@@ -50,6 +50,10 @@ def _load():
                                            pd, c_void_p, c_void_p, c_int64, p32]
         lib.oracle_argmax.argtypes = [pf, c_int64, c_int64, p32]
         lib.oracle_kv_rearrange.argtypes = [p16, p16, c_int, c_int, c_int, c_int, POINTER(c_uint8), p32]
+        lib.oracle_verify_attn_padded.argtypes = [p16, p16, p16, p16, p16, c_int, c_int, c_int, POINTER(c_uint8), c_int,
+                                                  p32, c_int, c_int, c_int, c_double, pd, c_void_p, p32]
+        lib.oracle_padded_append.argtypes = [p16, p16, c_int, c_int, c_int, c_int, POINTER(c_uint8), p32, p16, p16,
+                                             c_int, p32, p32, c_int, p32]
         lib.oracle_sample_targets.argtypes = [pf, p32, pf, c_int, c_int, c_int64, c_double, c_int64, c_float, p32]
         lib.oracle_accept.argtypes = [p32, p32, p32, c_int, c_int, c_int, p32, p32, p32, p32]
         lib.oracle_kv_commit.argtypes = [p16, p16, c_int, c_int, c_int, c_int, p32, c_int, p32, c_int,
@@ -152,6 +156,44 @@ def kv_rearrange(k, v, valid):
     _load().oracle_kv_rearrange(_ptr(k, c_uint16), _ptr(v, c_uint16), B, Hkv, cap, D, _ptr(valid, c_uint8),
                                 _ptr(lengths, c_int32))
     return {"k": k, "v": v, "valid": valid, "lengths": lengths}
+
+
+def verify_attn_padded(q, k_tree, v_tree, k, v, valid, extent: int, parent, scale, want_lse: bool = False):
+    """Sec. 3.2 attention over the padded batch cache of Sec. 4.3: k, v [B, Hkv, cap, D] (uint16 bf16
+    bits), valid [B, cap] u8, common length `extent`.  Returns dict(out, status[, lse])."""
+    q, k_tree, v_tree = _c(q, np.uint16), _c(k_tree, np.uint16), _c(v_tree, np.uint16)
+    k, v, valid, parent = _c(k, np.uint16), _c(v, np.uint16), _c(valid, np.uint8), _c(parent, np.int32)
+    B, T, Hq, D = q.shape
+    _, Hkv, cap, _ = k.shape
+    assert k.shape == (B, Hkv, cap, D) and v.shape == k.shape and valid.shape == (B, cap)
+    assert k_tree.shape == (B, T, Hkv, D) and v_tree.shape == k_tree.shape and parent.shape == (B, T)
+    out = np.zeros((B, T, Hq, D), dtype=np.float64)
+    lse = np.zeros((B, T, Hq), dtype=np.float64) if want_lse else None
+    status = np.zeros(B, dtype=np.int32)
+    _load().oracle_verify_attn_padded(
+        _ptr(q, c_uint16), _ptr(k_tree, c_uint16), _ptr(v_tree, c_uint16), _ptr(k, c_uint16), _ptr(v, c_uint16),
+        cap, Hkv, D, _ptr(valid, c_uint8), int(extent), _ptr(parent, c_int32), B, T, Hq, float(scale),
+        _ptr(out, c_double), lse.ctypes.data if lse is not None else None, _ptr(status, c_int32))
+    res = {"out": out, "status": status}
+    if want_lse:
+        res["lse"] = lse
+    return res
+
+
+def padded_append(k, v, valid, extent: int, k_tree, v_tree, path, n_acc):
+    """One step's growth of the padded batch cache (Sec. 4.3), on copies: the accepted rows behind the
+    common length, zero rows up to the batch's longest span.  Returns dict(k, v, valid, extent, status)."""
+    k, v, valid = _c(k, np.uint16).copy(), _c(v, np.uint16).copy(), _c(valid, np.uint8).copy()
+    k_tree, v_tree = _c(k_tree, np.uint16), _c(v_tree, np.uint16)
+    path, n_acc = _c(path, np.int32), _c(n_acc, np.int32)
+    B, Hkv, cap, D = k.shape
+    T = k_tree.shape[1]
+    ext = np.array([extent], dtype=np.int32)
+    status = np.zeros(B, dtype=np.int32)
+    _load().oracle_padded_append(_ptr(k, c_uint16), _ptr(v, c_uint16), B, Hkv, cap, D, _ptr(valid, c_uint8),
+                                 _ptr(ext, c_int32), _ptr(k_tree, c_uint16), _ptr(v_tree, c_uint16), T,
+                                 _ptr(path, c_int32), _ptr(n_acc, c_int32), path.shape[1], _ptr(status, c_int32))
+    return {"k": k, "v": v, "valid": valid, "extent": int(ext[0]), "status": status}
 
 
 def sample_targets(logits, parent, uniforms, temperature: float, top_k: int = 0, top_p: float = 1.0) -> np.ndarray:

@@ -19,6 +19,10 @@
  *                           drafted tokens, keep the longest consistent prefix.
  *   oracle_kv_rearrange     Sec. 4.3, Algorithm 4 on the padded batch cache:
  *                           internal padding removed, entries concatenated.
+ *   oracle_verify_attn_padded / oracle_padded_append
+ *                           Sec. 4.3, the padded batch cache itself: attention under
+ *                           its validity mask, and its growth by the batch's longest
+ *                           accepted span per step.
  *   oracle_sample_targets   Appendix C, randomized decoding: x* = F(P, U_t) with
  *                           coupled uniforms, temperature inverse-CDF sampling.
  *   oracle_kv_commit        Sec. 4.3 and Algorithm 4 (KVCacheRearrange): the
@@ -293,6 +297,132 @@ void oracle_kv_rearrange(uint16_t *k, uint16_t *v, int B, int Hkv, int cap, int 
         for (int t = 0; t < cap; ++t) valid[(size_t)b * cap + t] = t < n;
         lengths[b] = n;
     }
+}
+
+/*
+ * Sec. 4.3, the padded batch cache as the verification attention sees it (the layout the paper
+ * starts from, before and between rearrangements): k, v [B][Hkv][cap][D]; every sample's row is
+ * used up to the common length *extent; valid[b][t] != 0 marks a real entry, everything else
+ * is padding that no query may see.  For sample b, node j, query head h: softmax over the real
+ * entries t < extent in position order, then over the tree nodes on root..j (Sec. 3.2).
+ * A sample without any real entry attends over its tree path only.
+ * status: ORACLE_BAD_TREE per sample; ORACLE_CAPACITY for every sample when extent is outside
+ * [0, cap].  Rows of a rejected sample stay zero.
+ */
+void oracle_verify_attn_padded(const uint16_t *q, const uint16_t *k_tree, const uint16_t *v_tree,
+                               const uint16_t *k, const uint16_t *v, int cap, int n_kv_heads, int head_dim,
+                               const uint8_t *valid, int extent, const int32_t *parent, int batch,
+                               int n_nodes, int n_q_heads, double scale, double *out, double *lse,
+                               int32_t *status)
+{
+    const int G = n_q_heads / n_kv_heads;
+    const int D = head_dim;
+    memset(out, 0, sizeof(double) * (size_t)batch * n_nodes * n_q_heads * D);
+    if (lse) memset(lse, 0, sizeof(double) * (size_t)batch * n_nodes * n_q_heads);
+    for (int b = 0; b < batch; ++b) {
+        status[b] = ORACLE_OK;
+        if (extent < 0 || extent > cap) status[b] = ORACLE_CAPACITY;
+        else if (!oracle_tree_is_valid(parent + (size_t)b * n_nodes, n_nodes)) status[b] = ORACLE_BAD_TREE;
+    }
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < batch; ++b) {
+        for (int h = 0; h < n_q_heads; ++h) {
+            if (status[b] != ORACLE_OK) continue;
+            const int hk = h / G;
+            const int32_t *par = parent + (size_t)b * n_nodes;
+            double *score = (double *)malloc(sizeof(double) * (size_t)(extent + n_nodes));
+            const uint16_t **kptr = (const uint16_t **)malloc(sizeof(void *) * (size_t)(extent + n_nodes));
+            const uint16_t **vptr = (const uint16_t **)malloc(sizeof(void *) * (size_t)(extent + n_nodes));
+            for (int j = 0; j < n_nodes; ++j) {
+                const size_t row = ((size_t)b * n_nodes + j) * n_q_heads + h;
+                const uint16_t *qrow = q + row * D;
+                int n = 0;
+                for (int t = 0; t < extent; ++t) {
+                    if (!valid[(size_t)b * cap + t]) continue;
+                    const size_t at = (((size_t)b * n_kv_heads + hk) * cap + t) * D;
+                    kptr[n] = k + at;
+                    vptr[n] = v + at;
+                    ++n;
+                }
+                for (int i = j; i >= 0; i = par[i]) {
+                    const size_t at = (((size_t)b * n_nodes + i) * n_kv_heads + hk) * D;
+                    kptr[n] = k_tree + at;
+                    vptr[n] = v_tree + at;
+                    ++n;
+                }
+                double smax = -INFINITY;
+                for (int t = 0; t < n; ++t) {
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d)
+                        dot += bf16_bits_to_double(qrow[d]) * bf16_bits_to_double(kptr[t][d]);
+                    score[t] = scale * dot;
+                    if (score[t] > smax) smax = score[t];
+                }
+                double denom = 0.0;
+                for (int t = 0; t < n; ++t) {
+                    score[t] = exp(score[t] - smax);
+                    denom += score[t];
+                }
+                double *orow = out + row * D;
+                for (int t = 0; t < n; ++t) {
+                    const double p = score[t] / denom;
+                    for (int d = 0; d < D; ++d)
+                        orow[d] += p * bf16_bits_to_double(vptr[t][d]);
+                }
+                if (lse) lse[row] = smax + log(denom);
+            }
+            free(score);
+            free((void *)kptr);
+            free((void *)vptr);
+        }
+    }
+}
+
+/*
+ * Sec. 4.3, how the padded batch cache grows in one step: the accepted span of sample b (the K/V
+ * rows of path[b][0 .. n_acc[b]-1]) is written at positions extent .. extent + n_acc[b] - 1 of its
+ * row and marked real; the row is then filled with zero rows, marked padding, up to the batch's
+ * new common length extent + max_b n_acc[b] ("other prompts are padded with zeros to match the new
+ * maximum length").  *extent becomes that length.
+ * All or nothing: when the new length exceeds cap, or some n_acc is outside [0, max_path], or a
+ * path entry is not a node, every status is ORACLE_CAPACITY and nothing is changed.
+ */
+void oracle_padded_append(uint16_t *k, uint16_t *v, int B, int Hkv, int cap, int D, uint8_t *valid,
+                          int32_t *extent, const uint16_t *k_tree, const uint16_t *v_tree, int n_nodes,
+                          const int32_t *path, const int32_t *n_acc, int max_path, int32_t *status)
+{
+    const int E = *extent;
+    int grow = 0, ok = E >= 0 && E <= cap;
+    for (int b = 0; b < B; ++b) {
+        if (n_acc[b] < 0 || n_acc[b] > max_path) { ok = 0; continue; }
+        if (n_acc[b] > grow) grow = n_acc[b];
+        for (int i = 0; i < n_acc[b]; ++i) {
+            const int32_t node = path[(size_t)b * max_path + i];
+            if (node < 0 || node >= n_nodes) ok = 0;
+        }
+    }
+    if (ok && (int64_t)E + grow > cap) ok = 0;
+    for (int b = 0; b < B; ++b) status[b] = ok ? ORACLE_OK : ORACLE_CAPACITY;
+    if (!ok) return;
+    for (int b = 0; b < B; ++b) {
+        for (int i = 0; i < grow; ++i) {
+            const int t = E + i;
+            const int real = i < n_acc[b];
+            valid[(size_t)b * cap + t] = (uint8_t)real;
+            for (int h = 0; h < Hkv; ++h) {
+                const size_t dst = (((size_t)b * Hkv + h) * cap + t) * D;
+                if (real) {
+                    const size_t src = (((size_t)b * n_nodes + path[(size_t)b * max_path + i]) * Hkv + h) * D;
+                    memcpy(k + dst, k_tree + src, sizeof(uint16_t) * D);
+                    memcpy(v + dst, v_tree + src, sizeof(uint16_t) * D);
+                } else {
+                    memset(k + dst, 0, sizeof(uint16_t) * D);
+                    memset(v + dst, 0, sizeof(uint16_t) * D);
+                }
+            }
+        }
+    }
+    *extent = E + grow;
 }
 
 /*

@@ -379,3 +379,70 @@ def duplicate_shared_prefix(w: Workload) -> Workload:
     w2.k_pool, w2.v_pool, w2.page_table, w2.shared_prefix_len = k_pool, v_pool, pt, 0
     w2.name = w.name + "-dup"
     return w2
+
+
+@dataclass
+class PaddedCache:
+    """The padded batch cache of Sec. 4.3 (the layout the paper starts from)."""
+    k: np.ndarray        # u16 [B, Hkv, cap, D]
+    v: np.ndarray
+    valid: np.ndarray    # u8 [B, cap]
+    extent: int          # common length: no sample uses a row at or beyond it
+
+    @property
+    def capacity(self) -> int:
+        return int(self.k.shape[2])
+
+
+def padded_cache_of(w: Workload, seed: int, slack: int = 0, capacity: Optional[int] = None,
+                    fill_padding: int = 0) -> PaddedCache:
+    """The committed entries of workload `w` laid out as a padded batch cache: every sample's entries keep
+    their order but sit at a random sorted subset of the positions below the common extent
+    (= longest sample + `slack`), the other positions being padding.  Padding rows hold the bf16 bit
+    pattern `fill_padding` (0 = the paper's zeros); rows at or beyond the extent too."""
+    rng = np.random.default_rng(seed)
+    B, Hkv, D, P = w.batch, w.n_kv_heads, w.head_dim, w.page_size
+    lens = w.seq_lens.astype(np.int64)
+    extent = int(lens.max(initial=0)) + int(slack)
+    cap = int(capacity) if capacity is not None else extent
+    assert cap >= extent
+    k = np.full((B, Hkv, cap, D), fill_padding, np.uint16)
+    v = np.full((B, Hkv, cap, D), fill_padding, np.uint16)
+    valid = np.zeros((B, cap), np.uint8)
+    for b in range(B):
+        L = int(lens[b])
+        where = np.sort(rng.choice(extent, size=L, replace=False)) if L else np.zeros(0, np.int64)
+        pos = np.arange(L)
+        pg = w.page_table[b, pos // P]
+        k[b][:, where, :] = np.moveaxis(w.k_pool[pg, :, pos % P, :], 0, 1)
+        v[b][:, where, :] = np.moveaxis(w.v_pool[pg, :, pos % P, :], 0, 1)
+        valid[b, where] = 1
+    return PaddedCache(k=k, v=v, valid=valid, extent=extent)
+
+
+def accepted_spans(rng, batch: int, n_nodes: int, max_path: int, parent: np.ndarray, accept_rate: float,
+                   p_long: float):
+    """Accepted root paths of one step, drawn rather than verified (for cache-growth simulations):
+    the length is geometric in `accept_rate` (capped by the depth the tree offers) and, with
+    probability `p_long` per sample, the longest path of the tree up to max_path instead (a long
+    span proposed by the statistical search, Sec. 4.3).  Returns (path i32 [B, max_path], n_acc i32 [B]);
+    every path is a real root path of that sample's tree."""
+    path = np.zeros((batch, max_path), np.int32)
+    n_acc = np.zeros(batch, np.int32)
+    for b in range(batch):
+        par = parent[b]
+        lev = levels_of(par)
+        deepest = int(np.argmax(lev))                      # first node on the deepest level
+        chain = []
+        j = deepest
+        while j >= 0:
+            chain.append(j)
+            j = int(par[j])
+        chain = chain[::-1][:max_path]
+        if rng.random() < p_long:
+            n = len(chain)
+        else:
+            n = min(len(chain), int(rng.geometric(1.0 - accept_rate)))
+        n_acc[b] = n
+        path[b, :n] = chain[:n]
+    return path, n_acc
