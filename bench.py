@@ -601,6 +601,108 @@ def run_attn_table(args):
     rd.close()
 
 
+# ------------------------------------------------------------------------------------------------
+# the paper's padded batch cache against the paged cache over a run of decoding steps (Sec. 4.3)
+# ------------------------------------------------------------------------------------------------
+def run_cache_sim(args):
+    """Many verification steps with drawn accepted spans (geometric lengths, now and then a long span from
+    the statistical search): attention + cache maintenance per step, for the paged cache and for the padded
+    batch cache rearranged every N steps (Algorithm 4), N = 10, 25, 50 and never."""
+    import numpy as np
+    import torch
+    from paper_2508_09072_b200 import binding, workloads as W
+    torch.cuda.set_device(0)
+    rd = binding.Reader(0)
+    B, T, Hq, Hkv, D = 32, 32, 32, 8, 128
+    prompt, steps, chain, accept_rate, p_long = 1024, args.sim_steps, 16, 0.7, 0.03
+    max_path = chain
+    cap = -(-(prompt + steps * max_path) // 64) * 64
+    w = W.build_workload("cache-sim", 4242, [prompt] * B, T, Hq, Hkv, D,
+                         lambda r: W.widened_tree(r, T, chain, 6, 4), max_path=max_path, vocab=16, shuffle_pages=True,
+                         with_logits=False, room=steps * max_path)
+    rng = np.random.default_rng(4243)
+    spans = [W.accepted_spans(rng, B, T, max_path, w.parent, accept_rate, p_long) for _ in range(steps)]
+    paths = torch.from_numpy(np.stack([s[0] for s in spans])).cuda()
+    n_accs = torch.from_numpy(np.stack([s[1] for s in spans])).cuda()
+    grown = int(sum(int(s[1].max()) for s in spans))
+    real = np.stack([s[1] for s in spans]).sum(axis=0)
+
+    d = binding.to_device(w, with_logits=False)
+    anc, _, _ = rd.tree_encode(d.parent)
+    pc = W.padded_cache_of(w, seed=1, slack=0, capacity=cap)
+    cache = binding.padded_to_device(pc)
+    valid0, lens0 = cache.valid.clone(), d.cache.seq_lens.clone()
+    out_paged, out_padded = torch.empty_like(d.q), torch.empty_like(d.q)
+    st = torch.empty(B, dtype=torch.int32, device="cuda")
+    slots = torch.empty((B, max_path), dtype=torch.int32, device="cuda")
+    lengths = torch.empty(B, dtype=torch.int32, device="cuda")
+    ws = torch.empty(int(rd.lib.reader_padded_workspace_bytes(rd._h, B, T, Hq, Hkv, D, cap)), dtype=torch.uint8, device="cuda")
+    bad = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+
+    def run_paged():
+        d.cache.seq_lens.copy_(lens0)
+        a, b = mk(), mk()
+        a.record()
+        for s in range(steps):
+            rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out_paged, status=st, workspace=ws)
+            bad.add_(st.max())
+            rd.kv_commit(d.cache, d.k_tree, d.v_tree, paths[s], n_accs[s], slots=slots, status=st)
+            bad.add_(st.max())
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    def run_padded(every):
+        cache.valid.copy_(valid0)
+        cache.extent.fill_(prompt)
+        peak = torch.zeros(1, dtype=torch.int32, device="cuda")
+        a, b = mk(), mk()
+        a.record()
+        for s in range(steps):
+            rd.verify_attn_padded(d.q, d.k_tree, d.v_tree, cache, d.parent, w.scale, anc_mask=anc, out=out_padded, status=st,
+                                  workspace=ws)
+            bad.add_(st.max())
+            rd.padded_append(cache, d.k_tree, d.v_tree, paths[s], n_accs[s], status=st)
+            bad.add_(st.max())
+            torch.maximum(peak, cache.extent, out=peak)
+            if every and s % every == every - 1:
+                rd.padded_rearrange(cache, lengths)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b), int(peak.item()), int(cache.extent.item())
+
+    run_paged()                                               # warm-up: descriptors, caches, clocks
+    t_paged = sorted(run_paged() for _ in range(3))[1]
+    assert d.cache.seq_lens.cpu().numpy().tolist() == (prompt + real).tolist()
+    rows = []
+    for every in (10, 25, 50, 0):
+        run_padded(every)
+        res = sorted(run_padded(every) for _ in range(3))[1]
+        assert cache.valid.sum(dim=1).cpu().numpy().tolist() == (prompt + real).tolist()
+        rows.append({"rearrange_every": every or "never", "ms_total": res[0], "us_per_step": res[0] / steps * 1e3,
+                     "vs_paged": res[0] / t_paged, "peak_extent": res[1], "final_extent": res[2]})
+    # the two designs hold the same entries: one more verification on the final caches must agree
+    rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out_paged, status=st, workspace=ws)
+    rd.verify_attn_padded(d.q, d.k_tree, d.v_tree, cache, d.parent, w.scale, anc_mask=anc, out=out_padded, status=st, workspace=ws)
+    torch.cuda.synchronize()
+    diff = float((out_paged.float() - out_padded.float()).abs().max().item())
+    assert int(bad.item()) == 0 and diff <= 2e-2, (int(bad.item()), diff)
+    by_n = {r["rearrange_every"]: r["ms_total"] for r in rows}
+    print(json.dumps({
+        "cache_sim": "verify attention + cache maintenance per step: paged cache against the padded batch cache of Sec. 4.3",
+        "config": {"batch": B, "tree_nodes": T, "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": D, "prompt_len": prompt,
+                   "steps": steps, "accept_rate": accept_rate, "p_long_span": p_long, "long_span": chain,
+                   "p_some_sample_long": 1 - (1 - p_long) ** B, "capacity": cap,
+                   "l2": "no flush: each step reads more KV than the 126 MB L2 holds"},
+        "accepted_per_sample_per_step": float(real.mean() / steps), "common_growth_per_step": grown / steps,
+        "paged": {"ms_total": t_paged, "us_per_step": t_paged / steps * 1e3},
+        "padded": rows,
+        "rearrangement_gain_n25_vs_never": 1 - by_n[25] / by_n["never"],
+        "max_abs_diff_final_outputs": diff}))
+    rd.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -614,9 +716,13 @@ def main():
     ap.add_argument("--sweep-tree", action="store_true", help="measure the attention call for several tree sizes instead")
     ap.add_argument("--sweep-iters", type=int, default=15)
     ap.add_argument("--attn-table", action="store_true", help="verify attention alone on C1..C5 instead")
+    ap.add_argument("--cache-sim", action="store_true", help="paged cache against the paper's padded batch cache over many steps instead")
+    ap.add_argument("--sim-steps", type=int, default=200)
     args = ap.parse_args()
     if args.attn_table:
         run_attn_table(args)
+    elif args.cache_sim:
+        run_cache_sim(args)
     elif args.sweep_tree:
         run_sweep(args)
     elif args.impl == "reference":

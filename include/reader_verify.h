@@ -14,7 +14,9 @@
  *     reader_kv_commit     accepted K/V rows -> cache tail, seq_lens += n_acc    (Algorithm 4)
  *   and, beside these: reader_sample_targets (the sampling policies of Appendix C in place of the
  *   argmax), reader_kv_commit_layers (all layers of a model in one launch), reader_kv_rearrange
- *   (Algorithm 4 on the paper's padded cache layout), reader_accept_noalloc.
+ *   (Algorithm 4 on the paper's padded cache layout), reader_verify_attn_padded /
+ *   reader_padded_append / reader_padded_rearrange (the padded cache of Sec. 4.3 run as a cache, to be
+ *   measured against the paged one), reader_accept_noalloc.
  *
  * Conventions common to every call
  *   - Every pointer named below is a DEVICE pointer owned by the caller unless it says "host".
@@ -242,6 +244,68 @@ reader_status reader_kv_commit_layers(reader_ctx *ctx, const reader_kv_cache *ca
 reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t batch, int32_t n_kv_heads,
                                   int32_t capacity, int32_t head_dim, uint8_t *valid, int32_t *lengths_out,
                                   void *stream);
+
+/*
+ * The padded batch cache of Sec. 4.3 as a cache in its own right: the layout the paper starts from,
+ * kept here beside the paged cache so that the two designs can be run and measured against each
+ * other.  Every sample owns one row of `capacity` positions; all rows are in use up to the common
+ * length *extent; within a row real entries and padding alternate as the steps left them.
+ *   k, v      bf16 [batch][n_kv_heads][capacity][head_dim]
+ *   valid     u8   [batch][capacity]: non-zero marks a real entry; zero at and beyond *extent
+ *             (the two calls that move *extent keep it so; the attention ignores bytes there anyway)
+ *   extent    i32  [1] DEVICE scalar: rows at or beyond it are unused in every sample
+ * Padding rows may hold anything (the calls below write zeros there, as the paper does): no
+ * query ever sees them.
+ */
+typedef struct {
+    void *k;
+    void *v;
+    uint8_t *valid;
+    int32_t *extent;
+    int32_t capacity, n_kv_heads, head_dim;
+} reader_padded_cache;
+
+/* Workspace for reader_verify_attn_padded: that of reader_workspace_bytes plus the packed mask. */
+size_t reader_padded_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes,
+                                     int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                     int32_t capacity);
+
+/*
+ * reader_verify_attn (Sec. 3.2) over a padded batch cache: node j of sample b attends over the
+ * real entries of row b below *extent, in position order, and over the tree nodes on its root
+ * path.  Arguments, outputs, kernels and error channels are those of reader_verify_attn; there is
+ * no page table, and status_out[b] = READER_ERR_CAPACITY for every sample when *extent is outside
+ * [0, capacity].  Every sample costs the common length, padding included: that is the overhead
+ * Sec. 4.3 describes.  head_dim 64 or 128; k, v 16-byte aligned.
+ */
+reader_status reader_verify_attn_padded(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
+                                        const void *v_tree, const reader_padded_cache *cache,
+                                        const reader_tree *tree, float softmax_scale, void *out, float *lse_out,
+                                        void *workspace, size_t workspace_bytes, int32_t *status_out,
+                                        void *stream);
+
+/*
+ * One step's growth of a padded batch cache (Sec. 4.3: a long accepted span in one sample makes
+ * every other sample pad up to the new maximum length).  The K/V rows of path[b][0 .. n_acc[b]-1]
+ * are written at positions *extent .. *extent + n_acc[b] - 1 of row b and marked real; zero rows
+ * marked padding fill row b up to *extent + max_b n_acc[b], which becomes the new *extent.
+ *   k_tree, v_tree  bf16 [batch][n_nodes][n_kv_heads][head_dim];  path i32 [batch][max_path];
+ *   n_acc i32 [batch] (the outputs of reader_accept)
+ * All or nothing: when the new length exceeds capacity, an n_acc is outside [0, max_path] or a path
+ * entry is not a node, every status_out[b] is READER_ERR_CAPACITY and nothing is changed.
+ * head_dim a multiple of 8.
+ */
+reader_status reader_padded_append(reader_ctx *ctx, reader_padded_cache *cache, const void *k_tree,
+                                   const void *v_tree, int32_t batch, int32_t n_nodes, const int32_t *path,
+                                   const int32_t *n_acc, int32_t max_path, int32_t *status_out, void *stream);
+
+/*
+ * reader_kv_rearrange (Algorithm 4) on a reader_padded_cache, all `capacity` positions of it:
+ * afterwards every row is compact, lengths_out[b] (i32 [batch]) holds its entries and *extent is
+ * the longest of them.
+ */
+reader_status reader_padded_rearrange(reader_ctx *ctx, reader_padded_cache *cache, int32_t batch,
+                                      int32_t *lengths_out, void *stream);
 
 /*
  * reader_accept with target logits, for callers that cannot provide a workspace.  (The paper has

@@ -25,7 +25,8 @@ NOALLOC_MAX_ROWS = 4096
 EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
            "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
-           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers")
+           "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers",
+           "reader_padded_workspace_bytes", "reader_verify_attn_padded", "reader_padded_append", "reader_padded_rearrange")
 
 
 class ReaderError(RuntimeError):
@@ -38,6 +39,11 @@ class _KvCache(Structure):
     _fields_ = [("k_pool", c_void_p), ("v_pool", c_void_p), ("num_pages", c_int32), ("page_size", c_int32),
                 ("n_kv_heads", c_int32), ("head_dim", c_int32), ("page_table", c_void_p),
                 ("max_pages_per_seq", c_int32), ("seq_lens", c_void_p), ("shared_prefix_len", c_int32)]
+
+
+class _PaddedCache(Structure):
+    _fields_ = [("k", c_void_p), ("v", c_void_p), ("valid", c_void_p), ("extent", c_void_p), ("capacity", c_int32),
+                ("n_kv_heads", c_int32), ("head_dim", c_int32)]
 
 
 class _Tree(Structure):
@@ -91,6 +97,17 @@ def load_library() -> ctypes.CDLL:
     lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
                                         c_void_p, c_void_p]
     lib.reader_kv_rearrange.restype = c_int32
+    lib.reader_padded_workspace_bytes.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32]
+    lib.reader_padded_workspace_bytes.restype = c_size_t
+    lib.reader_verify_attn_padded.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, POINTER(_PaddedCache),
+                                              POINTER(_Tree), c_float, c_void_p, c_void_p, c_void_p, c_size_t,
+                                              c_void_p, c_void_p]
+    lib.reader_verify_attn_padded.restype = c_int32
+    lib.reader_padded_append.argtypes = [c_void_p, POINTER(_PaddedCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
+                                         c_void_p, c_int32, c_void_p, c_void_p]
+    lib.reader_padded_append.restype = c_int32
+    lib.reader_padded_rearrange.argtypes = [c_void_p, POINTER(_PaddedCache), c_int32, c_void_p, c_void_p]
+    lib.reader_padded_rearrange.restype = c_int32
     lib.reader_kv_commit.argtypes = [c_void_p, POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_int32, c_void_p,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
     lib.reader_kv_commit.restype = c_int32
@@ -131,6 +148,23 @@ class KvCache:
         n, h, p, d = self.k_pool.shape
         return _KvCache(self.k_pool.data_ptr(), self.v_pool.data_ptr(), n, p, h, d, self.page_table.data_ptr(),
                         self.page_table.shape[1], self.seq_lens.data_ptr(), int(self.shared_prefix_len))
+
+
+@dataclass
+class PaddedCache:
+    """The padded batch cache of Sec. 4.3; tensors live on the device and are owned by the caller."""
+    k: torch.Tensor        # bf16 [B, Hkv, capacity, D]
+    v: torch.Tensor
+    valid: torch.Tensor    # u8 [B, capacity]
+    extent: torch.Tensor   # i32 [1]: the common length
+
+    def _c(self) -> _PaddedCache:
+        _dev(self.k, torch.bfloat16, "k"); _dev(self.v, torch.bfloat16, "v")
+        _dev(self.valid, torch.uint8, "valid"); _dev(self.extent, torch.int32, "extent")
+        B, Hkv, cap, D = self.k.shape
+        if self.v.shape != self.k.shape or self.valid.shape != (B, cap) or self.extent.numel() != 1:
+            raise ValueError("padded cache: k, v [B, Hkv, cap, D], valid [B, cap], extent [1]")
+        return _PaddedCache(self.k.data_ptr(), self.v.data_ptr(), self.valid.data_ptr(), self.extent.data_ptr(), cap, Hkv, D)
 
 
 class Reader:
@@ -229,6 +263,58 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_verify_attn")
         return out, status
+
+    def verify_attn_padded(self, q: torch.Tensor, k_tree: torch.Tensor, v_tree: torch.Tensor, cache: PaddedCache,
+                           parent: torch.Tensor, scale: float, anc_mask: Optional[torch.Tensor] = None,
+                           out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                           status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+        """reader_verify_attn_padded: the same attention over the padded batch cache of Sec. 4.3."""
+        _dev(q, torch.bfloat16, "q"); _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        _dev(parent, torch.int32, "parent")
+        B, T, Hq, D = q.shape
+        Hkv = k_tree.shape[2]
+        c = cache._c()
+        out = out if out is not None else torch.empty_like(q)
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=q.device)
+        if workspace is None:
+            need = int(self.lib.reader_padded_workspace_bytes(self._h, max(B, 1), T, Hq, Hkv, D, c.capacity))
+            if need == 0:
+                raise ReaderError(ERR_INVALID_ARG, "reader_padded_workspace_bytes")
+            if self._ws is None or self._ws.numel() < need:
+                self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
+            workspace = self._ws
+        tree = _Tree(B, T, parent.data_ptr(), None if anc_mask is None else anc_mask.data_ptr())
+        st = self.lib.reader_verify_attn_padded(self._h, _ptr(q), Hq, _ptr(k_tree), _ptr(v_tree), ctypes.byref(c),
+                                                ctypes.byref(tree), float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                                workspace.numel(), _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_verify_attn_padded")
+        return out, status
+
+    def padded_append(self, cache: PaddedCache, k_tree: torch.Tensor, v_tree: torch.Tensor, path: torch.Tensor,
+                      n_acc: torch.Tensor, status: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """reader_padded_append: one step's accepted rows behind the common length, zero rows for the rest."""
+        _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        _dev(path, torch.int32, "path"); _dev(n_acc, torch.int32, "n_acc")
+        B, T = k_tree.shape[:2]
+        c = cache._c()
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=k_tree.device)
+        st = self.lib.reader_padded_append(self._h, ctypes.byref(c), _ptr(k_tree), _ptr(v_tree), B, T, _ptr(path), _ptr(n_acc),
+                                           path.shape[1] if path.dim() == 2 else 1, _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_padded_append")
+        return status
+
+    def padded_rearrange(self, cache: PaddedCache, lengths: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """reader_padded_rearrange: Algorithm 4 on the whole cache; the common length becomes the longest row."""
+        c = cache._c()
+        B = cache.k.shape[0]
+        if lengths is None:
+            lengths = torch.empty(B, dtype=torch.int32, device=cache.k.device)
+        st = self.lib.reader_padded_rearrange(self._h, ctypes.byref(c), B, _ptr(lengths), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_padded_rearrange")
+        return lengths
 
     def accept(self, parent: torch.Tensor, node_tokens: torch.Tensor, max_path: int,
                logits: Optional[torch.Tensor] = None, target_ids: Optional[torch.Tensor] = None,
@@ -390,3 +476,9 @@ def to_device(w, device="cuda:0", with_logits: bool = True) -> DeviceWorkload:
     return DeviceWorkload(bf16_tensor(w.q, device), bf16_tensor(w.k_tree, device), bf16_tensor(w.v_tree, device),
                           cache, torch.from_numpy(w.parent).to(device), torch.from_numpy(w.node_tokens).to(device),
                           logits, float(w.scale), int(w.max_path))
+
+
+def padded_to_device(pc, device="cuda:0") -> PaddedCache:
+    """A workloads.PaddedCache (numpy) as device tensors."""
+    return PaddedCache(bf16_tensor(pc.k, device), bf16_tensor(pc.v, device), torch.from_numpy(pc.valid).to(device),
+                       torch.tensor([pc.extent], dtype=torch.int32, device=device))

@@ -142,6 +142,79 @@ reader_status reader_tree_encode(reader_ctx *ctx, const int32_t *parent, int32_t
     return launch_status();
 }
 
+}  // extern "C"
+
+namespace {
+
+// What the two attention entry points share once their cache-specific arguments are checked: the
+// workspace is carved, the parameter block completed and the three kernels are enqueued.
+// `p` arrives with the cache fields set; `bits_offset` is where the packed mask of a padded cache
+// lives in the workspace (unused for the paged cache).
+reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cache *paged, const reader_padded_cache *padded,
+                              const reader_tree *tree, float softmax_scale, void *workspace, size_t workspace_bytes,
+                              void *stream) {
+    const int B = p.B, T = p.T, Hkv = p.Hkv, D = p.D;
+    const int n_mtiles = (T * p.G + kTileM - 1) / kTileM;
+    const int n_tree_tiles = (T + kPage - 1) / kPage;
+    const int64_t max_pages = padded ? ((int64_t)padded->capacity + kPage - 1) / kPage : paged->max_pages_per_seq;
+    const int64_t tiles_bound = (int64_t)B * Hkv * n_mtiles * (max_pages + n_tree_tiles + kUnitOverhead);
+    if (tiles_bound >= (int64_t)1 << 31) return READER_ERR_UNSUPPORTED;
+    if (n_mtiles > max_ctas(ctx)) return READER_ERR_UNSUPPORTED;   // a lane holds one CTA per M tile of a KV stream
+    const WsLayout w = ws_layout(ctx, B, T, D);
+    const size_t bits_bytes = padded ? align_up(sizeof(uint64_t) * (size_t)B * (size_t)max_pages) : 0;
+    if (workspace_bytes < w.total + bits_bytes) return READER_ERR_WORKSPACE;
+    if (reader_status st = check_device(ctx)) return st;
+
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = (cudaStream_t)stream;
+    p.anc = tree->anc_mask ? tree->anc_mask : reinterpret_cast<const uint64_t *>(ws + w.anc);
+    p.partial_o = reinterpret_cast<float *>(ws + w.partial_o);
+    p.partial_ml = reinterpret_cast<float *>(ws + w.partial_ml);
+    p.split_desc = reinterpret_cast<SplitDesc *>(ws + w.split_desc);
+    p.error_flag = reinterpret_cast<int32_t *>(ws + w.error_flag);
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.sched.seq_tile_start = reinterpret_cast<const int32_t *>(ws + w.seq_tile_start);
+    p.sched.seq_ntiles = reinterpret_cast<const int32_t *>(ws + w.seq_ntiles);
+    p.sched.seq_npages = reinterpret_cast<const int32_t *>(ws + w.seq_npages);
+    p.sched.units_per_seq = Hkv;
+    p.sched.n_mtiles = n_mtiles;
+    PaddedIn pin{};
+    reader_kv_cache none{};
+    if (padded) {
+        pin.valid = padded->valid;
+        pin.extent = padded->extent;
+        pin.cap = padded->capacity;
+        pin.bits = reinterpret_cast<uint64_t *>(ws + w.total);
+        pin.bits_per_seq = (int)max_pages;
+        p.valid_bits = pin.bits;
+        p.bits_per_seq = pin.bits_per_seq;
+        p.cap = padded->capacity;
+    }
+
+    const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
+    if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
+    const bool use_tc = tc_ok && ctx->attn_kernel != 1;
+    p.sched.n_ctas = max_ctas(ctx);   // two resident CTAs per SM for both kernels
+
+    launch_prepare(paged ? *paged : none, pin, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
+                   tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
+                   reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
+                   reinterpret_cast<int32_t *>(ws + w.seq_npages), p.status, p.error_flag, p.out, p.lse, p.Hq, D, st);
+    if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
+    if (use_tc) {
+        if (reader_status s = launch_attn_sm100(&ctx->sm100, p, st)) return s;
+    } else {
+        launch_attn_generic(p, st);
+    }
+    if (ctx->ev_stop) cudaEventRecord(ctx->ev_stop, st);
+    launch_combine(p, st);
+    return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
 reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
                                  const void *v_tree, const reader_kv_cache *cache, const reader_tree *tree,
                                  float softmax_scale, void *out, float *lse_out, void *workspace,
@@ -161,19 +234,6 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
         !aligned16(cache->v_pool) || !aligned16(out) || !aligned16(tree->anc_mask) ||
         (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0)
         return READER_ERR_INVALID_ARG;
-    const int G = Hq / Hkv;
-    const int n_mtiles = (T * G + kTileM - 1) / kTileM;
-    const int n_tree_tiles = (T + kPage - 1) / kPage;
-    const int64_t tiles_bound = (int64_t)B * Hkv * n_mtiles * ((int64_t)cache->max_pages_per_seq + n_tree_tiles);
-    if (tiles_bound >= (int64_t)1 << 31) return READER_ERR_UNSUPPORTED;
-    if (n_mtiles > max_ctas(ctx)) return READER_ERR_UNSUPPORTED;   // a lane holds one CTA per M tile of a KV stream
-    const WsLayout w = ws_layout(ctx, B, T, D);
-    if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
-    if (reader_status st = check_device(ctx)) return st;
-
-    unsigned char *ws = static_cast<unsigned char *>(workspace);
-    cudaStream_t st = (cudaStream_t)stream;
-
     AttnParams p{};
     p.q = static_cast<const __nv_bfloat16 *>(q);
     p.k_tree = static_cast<const __nv_bfloat16 *>(k_tree);
@@ -182,42 +242,81 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.v_pool = static_cast<const __nv_bfloat16 *>(cache->v_pool);
     p.page_table = cache->page_table;
     p.seq_lens = cache->seq_lens;
-    p.anc = tree->anc_mask ? tree->anc_mask : reinterpret_cast<const uint64_t *>(ws + w.anc);
     p.out = static_cast<__nv_bfloat16 *>(out);
     p.lse = lse_out;
-    p.partial_o = reinterpret_cast<float *>(ws + w.partial_o);
-    p.partial_ml = reinterpret_cast<float *>(ws + w.partial_ml);
-    p.split_desc = reinterpret_cast<SplitDesc *>(ws + w.split_desc);
     p.status = status_out;
-    p.error_flag = reinterpret_cast<int32_t *>(ws + w.error_flag);
-    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = G;
+    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
     p.max_pages = cache->max_pages_per_seq;
     p.num_pages = cache->num_pages;
+    p.pool_rows = (int64_t)cache->num_pages * Hkv * kPage;
     p.shared_prefix_pages = cache->shared_prefix_len / kPage;
-    p.scale_log2 = softmax_scale * 1.4426950408889634f;
-    p.sched.seq_tile_start = reinterpret_cast<const int32_t *>(ws + w.seq_tile_start);
-    p.sched.seq_ntiles = reinterpret_cast<const int32_t *>(ws + w.seq_ntiles);
-    p.sched.seq_npages = reinterpret_cast<const int32_t *>(ws + w.seq_npages);
-    p.sched.units_per_seq = Hkv;
-    p.sched.n_mtiles = n_mtiles;
+    return run_verify_attn(ctx, p, cache, nullptr, tree, softmax_scale, workspace, workspace_bytes, stream);
+}
 
-    const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
-    if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
-    const bool use_tc = tc_ok && ctx->attn_kernel != 1;
-    p.sched.n_ctas = max_ctas(ctx);   // two resident CTAs per SM for both kernels
+size_t reader_padded_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes, int32_t n_q_heads,
+                                     int32_t n_kv_heads, int32_t head_dim, int32_t capacity) {
+    if (!ctx || capacity < 1 || !shape_ok(max_batch, max_nodes, n_q_heads, n_kv_heads, head_dim)) return 0;
+    const size_t words = (size_t)max_batch * (((size_t)capacity + kPage - 1) / kPage);
+    return ws_layout(ctx, max_batch, max_nodes, head_dim).total + align_up(sizeof(uint64_t) * words);
+}
 
-    launch_prepare(*cache, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
-                   tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
-                   reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
-                   reinterpret_cast<int32_t *>(ws + w.seq_npages), status_out, p.error_flag, p.out, p.lse, Hq, D, st);
-    if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
-    if (use_tc) {
-        if (reader_status s = launch_attn_sm100(&ctx->sm100, p, *cache, st)) return s;
-    } else {
-        launch_attn_generic(p, st);
-    }
-    if (ctx->ev_stop) cudaEventRecord(ctx->ev_stop, st);
-    launch_combine(p, st);
+reader_status reader_verify_attn_padded(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
+                                        const void *v_tree, const reader_padded_cache *cache, const reader_tree *tree,
+                                        float softmax_scale, void *out, float *lse_out, void *workspace,
+                                        size_t workspace_bytes, int32_t *status_out, void *stream) {
+    if (!ctx || !cache || !tree) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;
+    if (!q || !k_tree || !v_tree || !out || !workspace || !status_out) return READER_ERR_INVALID_ARG;
+    const int B = tree->batch, T = tree->n_nodes, Hq = n_q_heads, Hkv = cache->n_kv_heads, D = cache->head_dim;
+    if (!cache->k || !cache->v || !cache->valid || !cache->extent || !tree->parent) return READER_ERR_INVALID_ARG;
+    if (B < 0 || T < 1 || T > kMaxNodes || Hq < 1 || Hkv < 1 || cache->capacity < 1 || !(softmax_scale == softmax_scale))
+        return READER_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128)) return READER_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k) || !aligned16(cache->v) ||
+        !aligned16(out) || !aligned16(tree->anc_mask) || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0)
+        return READER_ERR_INVALID_ARG;
+    AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.k_tree = static_cast<const __nv_bfloat16 *>(k_tree);
+    p.v_tree = static_cast<const __nv_bfloat16 *>(v_tree);
+    p.k_pool = static_cast<const __nv_bfloat16 *>(cache->k);
+    p.v_pool = static_cast<const __nv_bfloat16 *>(cache->v);
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse_out;
+    p.status = status_out;
+    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
+    p.pool_rows = (int64_t)B * Hkv * cache->capacity;
+    return run_verify_attn(ctx, p, nullptr, cache, tree, softmax_scale, workspace, workspace_bytes, stream);
+}
+
+reader_status reader_padded_append(reader_ctx *ctx, reader_padded_cache *cache, const void *k_tree, const void *v_tree,
+                                   int32_t batch, int32_t n_nodes, const int32_t *path, const int32_t *n_acc,
+                                   int32_t max_path, int32_t *status_out, void *stream) {
+    if (!ctx || !cache) return READER_ERR_INVALID_ARG;
+    if (batch == 0) return READER_OK;
+    if (!k_tree || !v_tree || !path || !n_acc || !status_out || !cache->k || !cache->v || !cache->valid || !cache->extent)
+        return READER_ERR_INVALID_ARG;
+    if (batch < 0 || n_nodes < 1 || n_nodes > kMaxNodes || max_path < 1 || cache->n_kv_heads < 1 || cache->capacity < 1)
+        return READER_ERR_INVALID_ARG;
+    if (cache->head_dim % 8 != 0 || cache->head_dim < 8) return READER_ERR_UNSUPPORTED;
+    if (!aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k) || !aligned16(cache->v)) return READER_ERR_INVALID_ARG;
+    if (reader_status st = check_device(ctx)) return st;
+    launch_padded_append(static_cast<__nv_bfloat16 *>(cache->k), static_cast<__nv_bfloat16 *>(cache->v), batch,
+                         cache->n_kv_heads, cache->capacity, cache->head_dim, cache->valid, cache->extent,
+                         static_cast<const __nv_bfloat16 *>(k_tree), static_cast<const __nv_bfloat16 *>(v_tree), n_nodes,
+                         path, n_acc, max_path, status_out, (cudaStream_t)stream);
+    return launch_status();
+}
+
+reader_status reader_padded_rearrange(reader_ctx *ctx, reader_padded_cache *cache, int32_t batch, int32_t *lengths_out,
+                                      void *stream) {
+    if (!ctx || !cache) return READER_ERR_INVALID_ARG;
+    if (batch == 0) return READER_OK;
+    if (!cache->extent || !lengths_out) return READER_ERR_INVALID_ARG;
+    const reader_status s = reader_kv_rearrange(ctx, cache->k, cache->v, batch, cache->n_kv_heads, cache->capacity,
+                                                cache->head_dim, cache->valid, lengths_out, stream);
+    if (s != READER_OK) return s;
+    launch_set_extent(lengths_out, batch, cache->extent, (cudaStream_t)stream);
     return launch_status();
 }
 

@@ -183,10 +183,33 @@ struct AttnParams {
     int32_t *error_flag;       // one word in the workspace: set on a bounded-wait timeout
     int B, T, Hq, Hkv, D, G;
     int max_pages, num_pages;
+    int64_t pool_rows;         // rows of head_dim elements in k_pool / v_pool (what a TMA descriptor may cover)
     int shared_prefix_pages;   // leading page-table entries common to every sequence
     float scale_log2;          // softmax_scale * log2(e)
+    // Padded batch cache (Sec. 4.3) instead of the paged one when valid_bits != nullptr: k_pool / v_pool
+    // are then [B][Hkv][cap][D], tile t of (b, h) starts at row (b * Hkv + h) * cap + t * kPage, there is
+    // no page table and no per-sequence length, and bit r of valid_bits[b * bits_per_seq + t] tells
+    // whether row t * kPage + r of sample b is a real entry (0 at and beyond the common extent).
+    const uint64_t *valid_bits;
+    int bits_per_seq, cap;
     Sched sched;
 };
+
+// Committed length of sequence b (unused, 0, with the padded cache: its tiles carry their own masks).
+__device__ __forceinline__ int committed_len(const AttnParams &p, int b) { return p.valid_bits ? 0 : p.seq_lens[b]; }
+
+// Keys of committed tile t of sequence b that its queries may see, bit r = key t * kPage + r.
+__device__ __forceinline__ uint64_t page_visible(const AttnParams &p, int b, int t, int L) {
+    if (p.valid_bits) return p.valid_bits[(size_t)b * p.bits_per_seq + t];
+    const int valid = L - t * kPage;
+    return valid >= kPage ? ~0ull : ((1ull << valid) - 1);
+}
+
+// First row of committed tile t of KV stream (b, h) in the [rows][D] view of a pool.
+__device__ __forceinline__ int64_t page_first_row(const AttnParams &p, int b, int h, int t, int page) {
+    if (p.valid_bits) return ((int64_t)b * p.Hkv + h) * p.cap + (int64_t)t * kPage;
+    return ((int64_t)page * p.Hkv + h) * kPage;
+}
 
 __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
@@ -216,10 +239,22 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // Host-side launchers (one per .cu file)
 void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int32_t *level,
                         int32_t *status, cudaStream_t st);
-void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
+// The padded batch cache as the preparation kernel sees it (valid == nullptr: the paged cache is used).
+struct PaddedIn {
+    const uint8_t *valid;     // [B][cap]
+    const int32_t *extent;    // device scalar: the common length
+    int cap;
+    uint64_t *bits;           // out: [B][bits_per_seq], the mask packed per tile, cleared from the extent on
+    int bits_per_seq;
+};
+void launch_prepare(const reader_kv_cache &c, const PaddedIn &padded, const int32_t *parent, int B, int T, int n_tree_tiles,
                     int units_per_seq, uint64_t *anc_out /*nullable*/, int32_t *seq_tile_start,
                     int32_t *seq_ntiles, int32_t *seq_npages, int32_t *status, int32_t *error_flag,
                     __nv_bfloat16 *out, float *lse /*nullable*/, int Hq, int D, cudaStream_t st);
+void launch_padded_append(__nv_bfloat16 *k, __nv_bfloat16 *v, int B, int Hkv, int cap, int D, uint8_t *valid,
+                          int32_t *extent, const __nv_bfloat16 *k_tree, const __nv_bfloat16 *v_tree, int T,
+                          const int32_t *path, const int32_t *n_acc, int max_path, int32_t *status, cudaStream_t st);
+void launch_set_extent(const int32_t *lengths, int B, int32_t *extent, cudaStream_t st);
 void launch_attn_generic(const AttnParams &p, cudaStream_t st);
 void launch_combine(const AttnParams &p, cudaStream_t st);
 void launch_argmax(const float *logits, int64_t rows, int64_t vocab, int splits, float *part_val,

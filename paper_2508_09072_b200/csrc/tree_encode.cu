@@ -35,8 +35,11 @@ void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int3
 // One CTA.  Each warp takes sequences b = warp, warp + 32, ...: checks the tree (encoding the
 // masks when asked), the committed length against the page table's capacity and every page id
 // in use; then warp 0 turns the per-sequence tile counts into the flat prefix the attention
-// kernels cut into CTA ranges.
-__global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict__ page_table,
+// kernels cut into CTA ranges.  With the padded batch cache (pd.valid != nullptr) there is no page
+// table: every sample has the common extent as its length, and the validity bytes below it are packed
+// into one 64-bit word per tile for the attention kernels.
+__global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
+                                                       const int32_t *__restrict__ page_table,
                                                        const int32_t *__restrict__ seq_lens, int max_pages,
                                                        int num_pages, const int32_t *__restrict__ parent, int B,
                                                        int T, int n_tree_tiles, int units_per_seq,
@@ -52,6 +55,35 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may set itself up meanwhile
     if (threadIdx.x == 0) *error_flag = 0;
+    const bool padded = pd.valid != nullptr;
+    const int extent = padded ? *pd.extent : 0;
+    const bool extent_ok = extent >= 0 && extent <= pd.cap;
+    if (padded && extent_ok) {
+        // 16 mask bytes -> 16 bits; pieces from the extent on (up to the end of its tile) read as zero
+        const int pieces = ((extent + kPage - 1) / kPage) * (kPage / 16);
+        const bool vec = (pd.cap % 16 == 0) && (reinterpret_cast<uintptr_t>(pd.valid) % 16 == 0);
+        for (int i = threadIdx.x; i < B * pieces; i += blockDim.x) {
+            const int b = i / pieces, c = i - b * pieces;
+            const int first = c * 16, n = min(16, extent - first);   // n <= 0: past the extent
+            uint32_t bits = 0;
+            if (n > 0) {
+                const uint8_t *src = pd.valid + (size_t)b * pd.cap + first;
+                if (vec) {
+                    const uint4 x = *reinterpret_cast<const uint4 *>(src);
+                    const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t m = __vcmpne4(w4[q], 0u) & 0x08040201u;
+                        bits |= ((m | (m >> 8) | (m >> 16) | (m >> 24)) & 0xfu) << (4 * q);
+                    }
+                } else {
+                    for (int r = 0; r < n; ++r) bits |= (src[r] != 0 ? 1u : 0u) << r;
+                }
+                if (n < 16) bits &= (1u << n) - 1u;
+            }
+            reinterpret_cast<uint16_t *>(pd.bits + (size_t)b * pd.bits_per_seq)[c] = (uint16_t)bits;
+        }
+    }
     for (int b = warp; b < B; b += 32) {
         for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];
         __syncwarp();
@@ -65,9 +97,12 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
                 anc_out[((size_t)b * T + j) * 2 + 1] = hi;
             }
         }
-        const int L = seq_lens[b];
+        const int L = padded ? extent : seq_lens[b];
         int npages = 0;
-        if (st == READER_OK) {
+        if (padded) {
+            if (!extent_ok) st = READER_ERR_CAPACITY;   // whatever the tree: no sample can be served
+            else if (st == READER_OK) npages = (L + kPage - 1) / kPage;
+        } else if (st == READER_OK) {
             if (L < 0 || (int64_t)L > (int64_t)max_pages * kPage) {
                 st = READER_ERR_CAPACITY;
             } else {
@@ -112,11 +147,11 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const int32_t *__restrict
     }
 }
 
-void launch_prepare(const reader_kv_cache &c, const int32_t *parent, int B, int T, int n_tree_tiles,
+void launch_prepare(const reader_kv_cache &c, const PaddedIn &padded, const int32_t *parent, int B, int T, int n_tree_tiles,
                     int units_per_seq, uint64_t *anc_out, int32_t *seq_tile_start, int32_t *seq_ntiles,
                     int32_t *seq_npages, int32_t *status, int32_t *error_flag, __nv_bfloat16 *out, float *lse,
                     int Hq, int D, cudaStream_t st) {
-    prepare_kernel<<<1, 1024, 0, st>>>(c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages, parent, B, T,
+    prepare_kernel<<<1, 1024, 0, st>>>(padded, c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages, parent, B, T,
                                        n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles,
                                        seq_npages, status, error_flag, out, lse, Hq, D);
 }

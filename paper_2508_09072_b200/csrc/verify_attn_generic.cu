@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kTileM) attn_generic_kernel(const AttnParams p
         const bool row_ok = grow < p.T * p.G;
         const int j = row_ok ? grow / p.G : 0;
         const int hq = sg.h * p.G + (row_ok ? grow % p.G : 0);
-        const int L = p.seq_lens[sg.b];
+        const int L = committed_len(p, sg.b);
 
         uint32_t qreg[D / 2];
         {
@@ -56,17 +56,16 @@ __global__ void __launch_bounds__(kTileM) attn_generic_kernel(const AttnParams p
             uint64_t vis;
             __syncthreads();
             if (t < sg.npages) {
-                const int page = p.page_table[(size_t)sg.b * p.max_pages + t];
-                const int valid = min(kPage, L - t * kPage);
-                const size_t base = ((size_t)page * p.Hkv + sg.h) * kPage * D;
+                const int page = p.valid_bits ? 0 : p.page_table[(size_t)sg.b * p.max_pages + t];
+                vis = page_visible(p, sg.b, t, L);
+                const size_t base = (size_t)page_first_row(p, sg.b, sg.h, t, page) * D;
                 const uint4 *ksrc = reinterpret_cast<const uint4 *>(p.k_pool + base);
                 const uint4 *vsrc = reinterpret_cast<const uint4 *>(p.v_pool + base);
                 for (int c = tid; c < kPage * kChunks; c += kTileM) {
-                    const bool in = (c / kChunks) < valid;
+                    const bool in = (vis >> (c / kChunks)) & 1ull;   // rows no query may see are never read
                     ks[c] = in ? ksrc[c] : make_uint4(0, 0, 0, 0);
                     vs[c] = in ? vsrc[c] : make_uint4(0, 0, 0, 0);
                 }
-                vis = valid >= 64 ? ~0ull : ((1ull << valid) - 1);
             } else {
                 const int kt = t - sg.npages;
                 for (int c = tid; c < kPage * kChunks; c += kTileM) {

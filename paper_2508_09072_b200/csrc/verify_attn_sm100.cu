@@ -124,8 +124,25 @@ __device__ __forceinline__ bool ready(uint32_t bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_test_wait(bar, parity));
 }
 
+// The cache kind is a compile-time choice (kPadded: the padded batch cache of Sec. 4.3, else the paged
+// cache), so that neither pays for the other's addressing.
+template <bool kPadded>
+__device__ __forceinline__ int len_of(const AttnParams &p, int b) {
+    if constexpr (kPadded) return 0; else return p.seq_lens[b];
+}
+template <bool kPadded>
+__device__ __forceinline__ uint64_t visible_of(const AttnParams &p, int b, int t, int L) {
+    if constexpr (kPadded) {
+        return p.valid_bits[(size_t)b * p.bits_per_seq + t];
+    } else {
+        const int valid = L - t * kPage;
+        return valid >= kPage ? ~0ull : ((1ull << valid) - 1);
+    }
+}
+
 // Walks the tiles of a CTA's range in order; the producer keeps one cursor for keys and one for
 // values.  Page ids are fetched 32 at a time (one per lane) and handed out by shuffle.
+template <bool kPadded>
 struct TileCursor {
     int w, w_end;       // flat position of the next segment
     Segment sg;
@@ -138,7 +155,8 @@ struct TileCursor {
     __device__ __forceinline__ void refill(const AttnParams &p, int lane) {
         cache_t0 = t;
         const int tt = t + lane;
-        cache_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
+        if constexpr (kPadded) cache_page = 0;
+        else cache_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
     }
     __device__ __forceinline__ void next_segment(const AttnParams &p, int cta, int lane) {
         active = false;
@@ -148,7 +166,7 @@ struct TileCursor {
             if (sg.tile_end > sg.tile_begin) { active = true; break; }
         }
         if (!active) return;
-        L = p.seq_lens[sg.b];
+        L = len_of<kPadded>(p, sg.b);
         t = sg.tile_begin;
         refill(p, lane);
     }
@@ -169,8 +187,8 @@ struct TileCursor {
 // one KV head from the tree tensor (rows past the tensor's end read as zero).  Rows past the
 // valid count may therefore hold anything; the score side masks them by selection and the value
 // side never multiplies them (see the MMA issuer).  Called by the whole producer warp.
-template <int D>
-__device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor &c, const CUtensorMap *pool_map,
+template <int D, bool kPadded>
+__device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor<kPadded> &c, const CUtensorMap *pool_map,
                                           const CUtensorMap *tree_map, uint32_t dst, uint32_t full, int lane,
                                           uint64_t stream_policy, int first_streamed_tile) {
     using C = Cfg<D>;
@@ -178,7 +196,9 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor 
     if (lane != 0) return;
     mbar_arrive_expect_tx(full, C::kTileBytes);
     if (c.t < c.sg.npages) {
-        const int row = (page * p.Hkv + c.sg.h) * kPage;
+        int row;
+        if constexpr (kPadded) row = (c.sg.b * p.Hkv + c.sg.h) * p.cap + c.t * kPage;
+        else row = (page * p.Hkv + c.sg.h) * kPage;
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf) {
             // a page that no other CTA will read again should not push reusable lines out of L2
@@ -192,7 +212,7 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor 
     }
 }
 
-template <int D>
+template <int D, bool kPadded>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                   const __grid_constant__ CUtensorMap ktmap, const __grid_constant__ CUtensorMap vtmap,
@@ -265,7 +285,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         // shared prefix the hint measured slightly slower, so it is left off there)
         const uint64_t stream_policy = l2_policy_evict_first();
         const int first_streamed_tile = (p.sched.n_mtiles == 1 && p.shared_prefix_pages == 0) ? 0 : 0x7fffffff;
-        TileCursor kc, vc;
+        TileCursor<kPadded> kc, vc;
         kc.init(p, cta, lane, w_begin, w_end);
         vc.init(p, cta, lane, w_begin, w_end);
         // the query tile of the next segment goes in as soon as the last score product of the
@@ -293,7 +313,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (kc.active) {
                 const int stage = kc.it % kStagesK;
                 if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStagesK) & 1) ^ 1)) {
-                    load_tile<D>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
+                    load_tile<D, kPadded>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     kc.advance(p, cta, lane);
                     moved = true;
@@ -302,7 +322,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (vc.active) {
                 const int stage = vc.it % kStagesV;
                 if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStagesV) & 1) ^ 1)) {
-                    load_tile<D>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
+                    load_tile<D, kPadded>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     vc.advance(p, cta, lane);
                     moved = true;
@@ -370,27 +390,66 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             const int n = sg.tile_end - sg.tile_begin;
             w += sg.span;
             if (n <= 0) continue;
-            const int L = p.seq_lens[sg.b];
+            const int L = len_of<kPadded>(p, sg.b);
+            uint64_t vis_next = 0;
+            if constexpr (kPadded) vis_next = sg.tile_begin < sg.npages ? visible_of<true>(p, sg.b, sg.tile_begin, L) : 0;
             for (int tl = 0; tl < n; ++tl, ++i) {
                 const int stage = i % kStagesV;
-                wait(bar(&bars->p_full[i & 1]), (i >> 1) & 1, abort_s, p.error_flag);
-                wait(bar(&bars->v_full[stage]), (i / kStagesV) & 1, abort_s, p.error_flag);
-                tc_fence_after();
-                const uint32_t vbase = sV + stage * C::kTileBytes;
-                // keys past the end of the sequence / tree: whole 16-key slices are not multiplied at
-                // all, the rest of the last slice is zeroed in place
                 const int t = sg.tile_begin + tl;
-                const int valid = t < sg.npages ? min(kPage, L - t * kPage) : min(kPage, p.T - (t - sg.npages) * kPage);
-                const int slices = (valid + 15) >> 4;
-                if (valid & 15) {
-                    constexpr int kChunks = D / 8;
-                    for (int idx = lane; idx < (slices * 16 - valid) * kChunks; idx += 32) {
-                        const int rr = valid + idx / kChunks, cc = idx % kChunks;
-                        const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
+                const uint32_t vbase = sV + stage * C::kTileBytes;
+                int slices;
+                if constexpr (kPadded) {
+                    // keys no query may see (padding rows anywhere in the tile, nodes past the tree's end) must
+                    // not reach the product, whatever bytes they hold: 16-key slices behind the last visible
+                    // key are not multiplied at all, invisible rows before it are zeroed in place
+                    uint64_t vis = vis_next;
+                    if (t >= sg.npages) {
+                        const int nodes = min(kPage, p.T - (t - sg.npages) * kPage);
+                        vis = nodes >= kPage ? ~0ull : ((1ull << nodes) - 1);
                     }
-                    fence_proxy_async();
-                    __syncwarp();
+                    if (t + 1 < sg.tile_end && t + 1 < sg.npages) vis_next = visible_of<true>(p, sg.b, t + 1, L);   // ahead of the waits
+                    slices = (64 - __clzll((long long)vis) + 15) >> 4;
+                    if (tl == 0 && slices == 0) slices = 1;   // the first product of a segment initialises O
+                    const uint64_t zero_rows = ~vis & (slices == 4 ? ~0ull : ((1ull << (slices * 16)) - 1));
+                    wait(bar(&bars->p_full[i & 1]), (i >> 1) & 1, abort_s, p.error_flag);
+                    wait(bar(&bars->v_full[stage]), (i / kStagesV) & 1, abort_s, p.error_flag);
+                    tc_fence_after();
+                    if (zero_rows) {
+                        constexpr int kChunks = D / 8;              // 16-byte pieces per row
+                        constexpr int kRowsPerPass = 32 / kChunks;  // rows a warp zeroes at once
+                        uint64_t left = zero_rows;
+                        while (left) {
+                            // lanes 0..kChunks-1 take the lowest row still to do, the next kChunks lanes the one after
+                            uint64_t mine = left;
+                            for (int q = 0; q < lane / kChunks && mine; ++q) mine &= mine - 1;
+                            if (mine) {
+                                const int rr = __ffsll((long long)mine) - 1, cc = lane % kChunks;
+                                const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
+                            }
+                            for (int q = 0; q < kRowsPerPass && left; ++q) left &= left - 1;
+                        }
+                        fence_proxy_async();
+                        __syncwarp();
+                    }
+                } else {
+                    wait(bar(&bars->p_full[i & 1]), (i >> 1) & 1, abort_s, p.error_flag);
+                    wait(bar(&bars->v_full[stage]), (i / kStagesV) & 1, abort_s, p.error_flag);
+                    tc_fence_after();
+                    // keys past the end of the sequence / tree: whole 16-key slices are not multiplied at
+                    // all, the rest of the last slice is zeroed in place
+                    const int valid = t < sg.npages ? min(kPage, L - t * kPage) : min(kPage, p.T - (t - sg.npages) * kPage);
+                    slices = (valid + 15) >> 4;
+                    if (valid & 15) {
+                        constexpr int kChunks = D / 8;
+                        for (int idx = lane; idx < (slices * 16 - valid) * kChunks; idx += 32) {
+                            const int rr = valid + idx / kChunks, cc = idx % kChunks;
+                            const uint32_t off = (cc >> 3) * C::kHalfRowsKV + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + off), "r"(0u) : "memory");
+                        }
+                        fence_proxy_async();
+                        __syncwarp();
+                    }
                 }
                 if (lane == 0) {
                     const uint64_t vd = descV + (uint64_t)((stage * C::kTileBytes) >> 4);
@@ -417,7 +476,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
             w += sg.span;
             if (sg.tile_end <= sg.tile_begin) continue;
-            const int L = p.seq_lens[sg.b];
+            const int L = len_of<kPadded>(p, sg.b);
             const int grow = sg.mt * kTileM + tid;
             const bool row_ok = grow < p.T * p.G;
             const int j = row_ok ? grow / p.G : 0;
@@ -432,10 +491,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
 
             float m_used = -INFINITY, l = 0.f;
             for (int t = sg.tile_begin; t < sg.tile_end; ++t, ++it) {
+                // (with a padded cache the mask comes from memory: the load is issued ahead of the wait below)
                 uint64_t vis;
                 if (t < sg.npages) {
-                    const int valid = L - t * kPage;
-                    vis = valid >= kPage ? ~0ull : ((1ull << valid) - 1);
+                    vis = visible_of<kPadded>(p, sg.b, t, L);
                 } else {
                     vis = (t - sg.npages) == 0 ? anc_lo : anc_hi;
                 }
@@ -591,7 +650,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D view of a pool: rows = num_pages * n_kv_heads * page_size, head_dim columns; box = 64 x 64.
+// 2-D view of a pool (or of a padded batch cache): all its rows of head_dim columns; box = 64 x 64.
 bool encode_pool_map(void *fn, CUtensorMap *map, const void *pool, int64_t rows, int D) {
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
@@ -674,29 +733,31 @@ void sm100_host_destroy(Sm100Host *h) {
 bool sm100_supports(const Sm100Host *h, const AttnParams &p, float softmax_scale) {
     if (!h->ready) return false;
     if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return false;   // the row maximum is taken before scaling
-    const int64_t rows = (int64_t)p.num_pages * p.Hkv * kPage;
+    const int64_t rows = p.pool_rows;
     if (p.G > kTileM || kTileM % p.G != 0) return false;   // a query tile is a box of whole nodes
     return (p.D == 64 || p.D == 128) && rows >= 1 && rows < ((int64_t)1 << 31);
 }
 
-reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_kv_cache &cache, cudaStream_t st) {
+reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t st) {
     if (!h->attr_set) {
-        if (cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess) {
             cudaGetLastError();
             return READER_ERR_CUDA;
         }
         h->attr_set = true;
     }
     Sm100Maps *m = h->maps;
-    const int64_t rows = (int64_t)cache.num_pages * cache.n_kv_heads * kPage;
-    if (m->k_pool != cache.k_pool || m->v_pool != cache.v_pool || m->rows != rows || m->D != p.D) {
-        if (!encode_pool_map(h->encode_tiled, &m->kmap, cache.k_pool, rows, p.D) ||
-            !encode_pool_map(h->encode_tiled, &m->vmap, cache.v_pool, rows, p.D)) {
+    const int64_t rows = p.pool_rows;
+    if (m->k_pool != p.k_pool || m->v_pool != p.v_pool || m->rows != rows || m->D != p.D) {
+        if (!encode_pool_map(h->encode_tiled, &m->kmap, p.k_pool, rows, p.D) ||
+            !encode_pool_map(h->encode_tiled, &m->vmap, p.v_pool, rows, p.D)) {
             m->rows = -1;
             return READER_ERR_CUDA;
         }
-        m->k_pool = cache.k_pool; m->v_pool = cache.v_pool; m->rows = rows; m->D = p.D;
+        m->k_pool = p.k_pool; m->v_pool = p.v_pool; m->rows = rows; m->D = p.D;
     }
     const int64_t nodes = (int64_t)p.B * p.T;
     if (m->k_tree != p.k_tree || m->v_tree != p.v_tree || m->nodes != nodes || m->tree_heads != p.Hkv || m->tree_D != p.D) {
@@ -724,9 +785,9 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, const reader_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = p.D == 128
-        ? cudaLaunchKernelEx(&cfg, attn_sm100_kernel<128>, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap)
-        : cudaLaunchKernelEx(&cfg, attn_sm100_kernel<64>, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
+    auto kernel = p.D == 128 ? (p.valid_bits ? attn_sm100_kernel<128, true> : attn_sm100_kernel<128, false>)
+                             : (p.valid_bits ? attn_sm100_kernel<64, true> : attn_sm100_kernel<64, false>);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return READER_ERR_CUDA;

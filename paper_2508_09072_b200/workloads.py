@@ -241,11 +241,12 @@ def build_workload(name: str, seed: int, seq_lens: Sequence[int], n_nodes: int, 
                    shuffle_pages: bool, shared_prefix_len: int = 0, zipf_tokens: bool = True,
                    peaked_key_fraction: float = 0.0, page_size: int = PAGE_SIZE,
                    with_logits: bool = True, duplicate_sibling: bool = False,
-                   spare_pages: int = 0) -> Workload:
+                   spare_pages: int = 0, room: Optional[int] = None) -> Workload:
     """Draw every input of a verification step from one seed.
 
     seq_lens are the committed lengths (a shared prefix included).  Each page-table row is given
-    room for ``L_b + max_path`` tokens so that a commit never overflows.  With a shared prefix
+    room for ``L_b + max_path`` tokens so that a commit never overflows (``L_b + room`` when `room`
+    is given: a run of many steps).  With a shared prefix
     the first ``shared_prefix_len / page_size`` entries of every row name the same pages, stored
     once.  ``peaked_key_fraction`` scales that share of the committed token positions' keys (all
     KV heads) by 4 before rounding.  ``duplicate_sibling`` copies one sibling's token onto another
@@ -258,7 +259,7 @@ def build_workload(name: str, seed: int, seq_lens: Sequence[int], n_nodes: int, 
     lens = np.asarray(seq_lens, dtype=np.int32)
     assert shared_prefix_len % P == 0 and (B == 0 or int(lens.min()) >= shared_prefix_len)
     n_prefix = shared_prefix_len // P
-    pages_per_seq = [-(-(int(L) + max_path) // P) for L in lens]
+    pages_per_seq = [-(-(int(L) + (max_path if room is None else int(room))) // P) for L in lens]
     max_pages = max(pages_per_seq) if B else 1
     private = [n - n_prefix for n in pages_per_seq]
     num_pages = n_prefix + int(sum(private)) + spare_pages
