@@ -689,16 +689,25 @@ bool encode_q_map(void *fn, CUtensorMap *map, const void *q, int B, int T, int H
 
 }  // namespace
 
-struct Sm100Maps {
+// Cached TMA descriptors.  A model calls the kernel once per layer and step with that layer's pools, so
+// the pool descriptors are kept for the last kPoolEntries distinct pools (round robin); the tree and query
+// tensors change with every call in a real decode loop and get one entry each.
+constexpr int kPoolEntries = 128;
+struct PoolMaps {
     const void *k_pool = nullptr, *v_pool = nullptr;
     int64_t rows = -1;
     int D = 0;
+    alignas(64) CUtensorMap kmap, vmap;
+};
+struct Sm100Maps {
+    PoolMaps pools[kPoolEntries];
+    int next_pool = 0;
     const void *k_tree = nullptr, *v_tree = nullptr;
     int64_t nodes = -1;
     int tree_heads = 0, tree_D = 0;
     const void *q = nullptr;
     int qB = -1, qT = 0, qHq = 0, qG = 0, qD = 0;
-    alignas(64) CUtensorMap kmap, vmap, ktmap, vtmap, qmap;
+    alignas(64) CUtensorMap ktmap, vtmap, qmap;
 };
 
 reader_status sm100_host_init(Sm100Host *h, int device) {
@@ -751,13 +760,19 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t 
     }
     Sm100Maps *m = h->maps;
     const int64_t rows = p.pool_rows;
-    if (m->k_pool != p.k_pool || m->v_pool != p.v_pool || m->rows != rows || m->D != p.D) {
-        if (!encode_pool_map(h->encode_tiled, &m->kmap, p.k_pool, rows, p.D) ||
-            !encode_pool_map(h->encode_tiled, &m->vmap, p.v_pool, rows, p.D)) {
-            m->rows = -1;
+    PoolMaps *pm = nullptr;
+    for (int i = 0; i < kPoolEntries && !pm; ++i) {
+        PoolMaps &e = m->pools[i];
+        if (e.k_pool == p.k_pool && e.v_pool == p.v_pool && e.rows == rows && e.D == p.D) pm = &e;
+    }
+    if (!pm) {
+        pm = &m->pools[m->next_pool];
+        m->next_pool = (m->next_pool + 1) % kPoolEntries;
+        pm->rows = -1;
+        if (!encode_pool_map(h->encode_tiled, &pm->kmap, p.k_pool, rows, p.D) ||
+            !encode_pool_map(h->encode_tiled, &pm->vmap, p.v_pool, rows, p.D))
             return READER_ERR_CUDA;
-        }
-        m->k_pool = p.k_pool; m->v_pool = p.v_pool; m->rows = rows; m->D = p.D;
+        pm->k_pool = p.k_pool; pm->v_pool = p.v_pool; pm->rows = rows; pm->D = p.D;
     }
     const int64_t nodes = (int64_t)p.B * p.T;
     if (m->k_tree != p.k_tree || m->v_tree != p.v_tree || m->nodes != nodes || m->tree_heads != p.Hkv || m->tree_D != p.D) {
@@ -787,7 +802,7 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t 
     cfg.numAttrs = 1;
     auto kernel = p.D == 128 ? (p.valid_bits ? attn_sm100_kernel<128, true> : attn_sm100_kernel<128, false>)
                              : (p.valid_bits ? attn_sm100_kernel<64, true> : attn_sm100_kernel<64, false>);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p, m->kmap, m->vmap, m->ktmap, m->vtmap, m->qmap);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p, pm->kmap, pm->vmap, m->ktmap, m->vtmap, m->qmap);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return READER_ERR_CUDA;

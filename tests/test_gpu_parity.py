@@ -505,6 +505,67 @@ def test_whole_step_captured_in_a_cuda_graph_replays_identically(rd):
     assert int(status.max()) == 0 and int(cst.max()) == 0
 
 
+def test_multi_layer_step_in_one_graph_matches_oracle_layer_by_layer(rd):
+    """The step of a model with several layers as one captured launch sequence: verify attention on every
+    layer's own cache and tree tensors, one acceptance, one commit into all layers.  Replayed, every
+    layer's attention output and every layer's pools must be what the oracle computes for that layer."""
+    from paper_2508_09072_b200 import binding
+    n_layers = 3
+    w = W.make("c3", reduced=True)
+    rng = np.random.default_rng(77)
+    layers = [(w.q, w.k_tree, w.v_tree, w.k_pool, w.v_pool)]
+    for _ in range(n_layers - 1):
+        layers.append(tuple(W.normal_bf16(rng, a.shape) for a in layers[0]))
+    d = binding.to_device(w)
+    B, T = w.batch, w.n_nodes
+    dev = [tuple(binding.bf16_tensor(a, "cuda") for a in lay) for lay in layers]
+    caches = [binding.KvCache(l[3], l[4], d.cache.page_table, d.cache.seq_lens, 0) for l in dev]
+    outs_attn = [torch.empty_like(d.q) for _ in range(n_layers)]
+    status = torch.empty((n_layers, B), dtype=torch.int32, device="cuda")
+    ws = rd.workspace(B, T, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    tgt = torch.empty((B, T), dtype=torch.int32, device="cuda")
+    acc = tuple(torch.empty(sh, dtype=torch.int32, device="cuda") for sh in ((B, w.max_path), (B,), (B,), (B,)))
+    slots = torch.empty((B, w.max_path), dtype=torch.int32, device="cuda")
+    cst = torch.empty(B, dtype=torch.int32, device="cuda")
+    seq0 = d.cache.seq_lens.clone()
+
+    def step():
+        d.cache.seq_lens.copy_(seq0)
+        for l in range(n_layers):
+            rd.verify_attn(dev[l][0], dev[l][1], dev[l][2], caches[l], d.parent, w.scale, out=outs_attn[l], status=status[l],
+                           workspace=ws)
+        rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=tgt, workspace=ws, outs=acc)
+        rd.kv_commit_layers(caches, [l[1] for l in dev], [l[2] for l in dev], acc[0], acc[1], slots=slots, status=cst)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()                                   # first use on this stream happens outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for t in outs_attn + [tgt, slots]:
+        t.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.max()) == 0 and int(cst.max()) == 0
+    ref_acc = oracle.accept(w.parent, w.node_tokens, oracle.argmax(w.logits), w.max_path)
+    np.testing.assert_array_equal(acc[0].cpu().numpy(), ref_acc["path"])
+    np.testing.assert_array_equal(acc[1].cpu().numpy(), ref_acc["n_acc"])
+    for l, (q, kt, vt, kp, vp) in enumerate(layers):
+        ref = oracle.verify_attn(q, kt, vt, kp, vp, w.page_table, w.seq_lens, w.parent, w.scale)
+        got = W.bf16_bits_to_f32(binding.bf16_bits(outs_attn[l])).astype(np.float64)
+        err = np.abs(got - ref["out"])
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (l, err.max(), err.mean())
+        com = oracle.kv_commit(kp, vp, w.page_table, w.seq_lens, 0, kt, vt, ref_acc["path"], ref_acc["n_acc"])
+        np.testing.assert_array_equal(binding.bf16_bits(caches[l].k_pool), com["k_pool"])
+        np.testing.assert_array_equal(binding.bf16_bits(caches[l].v_pool), com["v_pool"])
+        np.testing.assert_array_equal(d.cache.seq_lens.cpu().numpy(), com["seq_lens"])
+        np.testing.assert_array_equal(slots.cpu().numpy(), com["slots"])
+
+
 def test_thousands_of_calls_never_hit_a_bounded_wait(rd):
     """Every device-side wait is bounded, so a lost wake-up shows as READER_ERR_TIMEOUT in the status
     words of one call in many (and as a one-second stall) rather than as a hang.  The status maximum
