@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "verified tree-tokens/s (verify attention + acceptance + KV commit, 1 step)"
 UNIT = "tokens/s"
-LAUNCHES_PER_STEP = 6   # prepare, attention, combine, argmax, accept walk, commit
+LAUNCHES_PER_STEP = 5   # prepare, attention, combine, argmax, acceptance walk + commit
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised under
 # profiles/ (C3 only); None when the kernel has changed since its counters were taken.
 NCU_TRAFFIC = {("verify_attn", "c3"): 328.9e6, ("accept (target argmax)", "c3"): 525.7e6}
@@ -235,11 +235,10 @@ def run_ours(args):
         rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=out, status=status, workspace=ws)
         if ev:
             ev[1].record()
-        rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=tgt, workspace=ws, outs=acc_out)
+        rd.accept_commit(d.parent, d.node_tokens, w.max_path, d.cache, d.k_tree, d.v_tree, logits=d.logits, target_ids=tgt,
+                         workspace=ws, outs=acc_out, slots=slots, commit_status=cstat)
         if ev:
             ev[2].record()
-        rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc_out[0], acc_out[1], slots=slots, status=cstat)
-        if ev:
             ev[3].record()
 
     def barrier():
@@ -506,8 +505,8 @@ def run_ours(args):
                             "tokens_per_s_call": tokens / (t_attn_call * 1e-3)},
             "accept": {"ms": t_argmax_kernel, "call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
                        "gbs": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9,
-                       "note": "ms / gbs: the argmax kernel alone; call_ms adds the acceptance walk"},
-            "kv_commit": {"call_ms": t_commit},
+                       "note": "ms / gbs: the argmax kernel alone; call_ms is reader_accept_commit: it adds the acceptance walk "
+                               "and the KV commit, which share one launch"},
             "kv_commit_32_layers": {"call_ms": t_layers, "note": "the accepted rows committed into 32 layers: 32 calls of "
                                     "reader_kv_commit against one reader_kv_commit_layers; not in the step"},
             "kv_rearrange": {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,

@@ -13,7 +13,8 @@
  *     reader_accept        target argmax + longest consistent root path          (Algorithm 5)
  *     reader_kv_commit     accepted K/V rows -> cache tail, seq_lens += n_acc    (Algorithm 4)
  *   and, beside these: reader_sample_targets (the sampling policies of Appendix C in place of the
- *   argmax), reader_kv_commit_layers (all layers of a model in one launch), reader_kv_rearrange
+ *   argmax), reader_accept_commit (acceptance and commit in one launch), reader_kv_commit_layers (all
+ *   layers of a model in one launch), reader_kv_rearrange
  *   (Algorithm 4 on the paper's padded cache layout), reader_verify_attn_padded /
  *   reader_padded_append / reader_padded_rearrange (the padded cache of Sec. 4.3 run as a cache, to be
  *   measured against the paged one), reader_accept_noalloc.
@@ -215,6 +216,21 @@ reader_status reader_kv_commit(reader_ctx *ctx, reader_kv_cache *cache, const vo
                                const int32_t *path, const int32_t *n_acc, int32_t max_path,
                                int32_t update_seq_lens, int32_t *slots_out, int32_t *status_out,
                                void *stream);
+
+/*
+ * reader_accept followed by reader_kv_commit for one layer, with the acceptance walk and the commit
+ * in a single launch (Algorithm 5, then Sec. 4.3 / Algorithm 4 in per-step form): one dependent
+ * launch fewer per decoding step.  Arguments and results are those of the two calls: status_out is
+ * reader_accept's status word, commit_status_out reader_kv_commit's; path_out and n_acc_out are both
+ * outputs of the walk and what is committed.
+ */
+reader_status reader_accept_commit(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens,
+                                   const float *logits, int32_t vocab, int32_t *target_ids, int32_t max_path,
+                                   reader_kv_cache *cache, const void *k_tree, const void *v_tree,
+                                   int32_t update_seq_lens, int32_t *path_out, int32_t *n_acc_out,
+                                   int32_t *bonus_out, int32_t *slots_out, void *workspace,
+                                   size_t workspace_bytes, int32_t *status_out, int32_t *commit_status_out,
+                                   void *stream);
 
 /*
  * reader_kv_commit for every layer of a model in one launch (the accepted path is the same in all

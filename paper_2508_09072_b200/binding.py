@@ -26,7 +26,7 @@ EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_se
            "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
            "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers",
-           "reader_padded_workspace_bytes", "reader_verify_attn_padded", "reader_padded_append", "reader_padded_rearrange")
+           "reader_accept_commit", "reader_padded_workspace_bytes", "reader_verify_attn_padded", "reader_padded_append", "reader_padded_rearrange")
 
 
 class ReaderError(RuntimeError):
@@ -97,6 +97,10 @@ def load_library() -> ctypes.CDLL:
     lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
                                         c_void_p, c_void_p]
     lib.reader_kv_rearrange.restype = c_int32
+    lib.reader_accept_commit.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
+                                         POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p,
+                                         c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p]
+    lib.reader_accept_commit.restype = c_int32
     lib.reader_padded_workspace_bytes.argtypes = [c_void_p, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32]
     lib.reader_padded_workspace_bytes.restype = c_size_t
     lib.reader_verify_attn_padded.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, POINTER(_PaddedCache),
@@ -344,6 +348,45 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_accept")
         return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids}
+
+    def accept_commit(self, parent: torch.Tensor, node_tokens: torch.Tensor, max_path: int, cache: KvCache,
+                      k_tree: torch.Tensor, v_tree: torch.Tensor, logits: Optional[torch.Tensor] = None,
+                      target_ids: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, outs=None,
+                      slots: Optional[torch.Tensor] = None, commit_status: Optional[torch.Tensor] = None,
+                      update_seq_lens: bool = True):
+        """reader_accept_commit: accept() and kv_commit() with the walk and the commit in one launch.
+        Returns a dict: path, n_acc, bonus, status, target_ids, slots, commit_status."""
+        _dev(parent, torch.int32, "parent"); _dev(node_tokens, torch.int32, "node_tokens")
+        _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        B, T = parent.shape
+        dev = parent.device
+        vocab = 0
+        if logits is not None:
+            _dev(logits, torch.float32, "logits")
+            vocab = logits.shape[-1]
+            if target_ids is None:
+                target_ids = torch.empty((B, T), dtype=torch.int32, device=dev)
+        elif target_ids is None:
+            raise TypeError("accept_commit: give logits or target_ids")
+        _dev(target_ids, torch.int32, "target_ids")
+        if outs is None:
+            outs = (torch.empty((B, max_path), dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev))
+        path, n_acc, bonus, status = outs
+        slots = slots if slots is not None else torch.empty((B, max_path), dtype=torch.int32, device=dev)
+        commit_status = commit_status if commit_status is not None else torch.empty(B, dtype=torch.int32, device=dev)
+        ws = workspace if workspace is not None else self.workspace(max(B, 1), T, 1, 1, 64)
+        tree = _Tree(B, T, parent.data_ptr(), None)
+        c = cache._c()
+        st = self.lib.reader_accept_commit(self._h, ctypes.byref(tree), _ptr(node_tokens), _ptr(logits), vocab,
+                                           _ptr(target_ids), int(max_path), ctypes.byref(c), _ptr(k_tree), _ptr(v_tree),
+                                           int(bool(update_seq_lens)), _ptr(path), _ptr(n_acc), _ptr(bonus), _ptr(slots),
+                                           _ptr(ws), ws.numel(), _ptr(status), _ptr(commit_status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_accept_commit")
+        return {"path": path, "n_acc": n_acc, "bonus": bonus, "status": status, "target_ids": target_ids,
+                "slots": slots, "commit_status": commit_status}
 
     def accept_noalloc(self, parent: torch.Tensor, node_tokens: torch.Tensor, max_path: int, logits: torch.Tensor,
                        target_ids: Optional[torch.Tensor] = None, outs=None):

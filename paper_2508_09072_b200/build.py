@@ -11,7 +11,7 @@ INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libreader_verify.so")
 
 SOURCES = ["api.cu", "tree_encode.cu", "verify_attn_generic.cu", "verify_attn_sm100.cu", "combine.cu",
-           "accept.cu", "accept_noalloc.cu", "sample.cu", "kv_commit.cu", "kv_rearrange.cu", "padded_cache.cu"]
+           "accept.cu", "accept_noalloc.cu", "sample.cu", "kv_commit.cu", "kv_rearrange.cu", "padded_cache.cu", "accept_commit.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "-I", INCLUDE, "-I", CSRC]

@@ -52,6 +52,16 @@ inline reader_status check_device(const reader_ctx *ctx) {
     return dev == ctx->device ? READER_OK : READER_ERR_INVALID_ARG;
 }
 
+// Column ranges a logits row is cut into so that small batches still fill the GPU (>= 2048 columns each).
+inline int argmax_splits(const reader_ctx *ctx, int64_t rows, int64_t vocab) {
+    int64_t want = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;
+    const int64_t cap = vocab / 2048 > 0 ? vocab / 2048 : 1;
+    if (want < 1) want = 1;
+    if (want > cap) want = cap;
+    if (want > kMaxSplits) want = kMaxSplits;
+    return (int)want;
+}
+
 inline reader_status launch_status() { return cudaGetLastError() == cudaSuccess ? READER_OK : READER_ERR_CUDA; }
 
 }  // namespace
@@ -343,11 +353,7 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
         const WsLayout w = ws_layout(ctx, B, T, 64);
         if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
         const int64_t rows = (int64_t)B * T;
-        int64_t want = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;
-        int64_t cap = vocab / 2048 > 0 ? vocab / 2048 : 1;
-        splits = (int)(want < 1 ? 1 : want);
-        if (splits > cap) splits = (int)cap;
-        if (splits > kMaxSplits) splits = kMaxSplits;
+        splits = argmax_splits(ctx, rows, vocab);
         unsigned char *ws = static_cast<unsigned char *>(workspace);
         pv = reinterpret_cast<float *>(ws + w.amax_val);
         pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);
@@ -357,6 +363,47 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
     }
     launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, pv, pi, splits, path_out, n_acc_out,
                   bonus_out, status_out, st);
+    return launch_status();
+}
+
+reader_status reader_accept_commit(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens, const float *logits,
+                                   int32_t vocab, int32_t *target_ids, int32_t max_path, reader_kv_cache *cache,
+                                   const void *k_tree, const void *v_tree, int32_t update_seq_lens, int32_t *path_out,
+                                   int32_t *n_acc_out, int32_t *bonus_out, int32_t *slots_out, void *workspace,
+                                   size_t workspace_bytes, int32_t *status_out, int32_t *commit_status_out, void *stream) {
+    if (!ctx || !tree || !cache) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;
+    if (!tree->parent || !node_tokens || !target_ids || !path_out || !n_acc_out || !bonus_out || !slots_out || !status_out ||
+        !commit_status_out || !k_tree || !v_tree || !cache->k_pool || !cache->v_pool || !cache->page_table || !cache->seq_lens)
+        return READER_ERR_INVALID_ARG;
+    const int B = tree->batch, T = tree->n_nodes;
+    if (B < 0 || T < 1 || T > kMaxNodes || max_path < 1 || cache->n_kv_heads < 1 || cache->max_pages_per_seq < 1 ||
+        cache->num_pages < 0 || cache->shared_prefix_len < 0 || cache->shared_prefix_len % kPage != 0)
+        return READER_ERR_INVALID_ARG;
+    if (cache->page_size != kPage || cache->head_dim % 8 != 0 || cache->head_dim < 8) return READER_ERR_UNSUPPORTED;
+    if (!aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k_pool) || !aligned16(cache->v_pool))
+        return READER_ERR_INVALID_ARG;
+    if (reader_status st = check_device(ctx)) return st;
+    cudaStream_t st = (cudaStream_t)stream;
+    int splits = 0;
+    float *pv = nullptr;
+    int32_t *pi = nullptr;
+    if (logits) {
+        if (vocab < 1 || !workspace || !aligned16(logits) || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0)
+            return READER_ERR_INVALID_ARG;
+        const WsLayout w = ws_layout(ctx, B, T, 64);
+        if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
+        splits = argmax_splits(ctx, (int64_t)B * T, vocab);
+        unsigned char *ws = static_cast<unsigned char *>(workspace);
+        pv = reinterpret_cast<float *>(ws + w.amax_val);
+        pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);
+        if (ctx->ev_acc_start) cudaEventRecord(ctx->ev_acc_start, st);
+        launch_argmax(logits, (int64_t)B * T, vocab, splits, pv, pi, st);
+        if (ctx->ev_acc_stop) cudaEventRecord(ctx->ev_acc_stop, st);
+    }
+    launch_accept_commit(tree->parent, node_tokens, target_ids, B, T, max_path, pv, pi, splits, path_out, n_acc_out, bonus_out,
+                         status_out, *cache, static_cast<const __nv_bfloat16 *>(k_tree), static_cast<const __nv_bfloat16 *>(v_tree),
+                         update_seq_lens, slots_out, commit_status_out, st);
     return launch_status();
 }
 

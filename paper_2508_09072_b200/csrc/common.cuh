@@ -267,6 +267,11 @@ void launch_kv_rearrange(__nv_bfloat16 *k, __nv_bfloat16 *v, int B, int Hkv, int
 void launch_accept(const int32_t *parent, const int32_t *tok, int32_t *target, int B, int T,
                    int max_path, const float *part_val, const int32_t *part_idx, int splits,
                    int32_t *path, int32_t *n_acc, int32_t *bonus, int32_t *status, cudaStream_t st);
+void launch_accept_commit(const int32_t *parent, const int32_t *tok, int32_t *target, int B, int T, int max_path,
+                          const float *part_val, const int32_t *part_idx, int splits, int32_t *path, int32_t *n_acc,
+                          int32_t *bonus, int32_t *status, const reader_kv_cache &c, const __nv_bfloat16 *k_tree,
+                          const __nv_bfloat16 *v_tree, int update_seq_lens, int32_t *slots, int32_t *commit_status,
+                          cudaStream_t st);
 // Pool and tree pointers of up to kCommitLayersPerLaunch layers, passed to the kernel by value.
 constexpr int kCommitLayersPerLaunch = 32;
 struct CommitLayers {

@@ -53,7 +53,8 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
                                                        int Hq, int D) {
     __shared__ int32_t par[32][kMaxNodes];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may set itself up meanwhile
+    pdl_launch_dependents();   // the attention kernel may set itself up meanwhile
+    pdl_wait();                // this kernel itself is launched ahead of its predecessor's end
     if (threadIdx.x == 0) *error_flag = 0;
     const bool padded = pd.valid != nullptr;
     const int extent = padded ? *pd.extent : 0;
@@ -151,9 +152,9 @@ void launch_prepare(const reader_kv_cache &c, const PaddedIn &padded, const int3
                     int units_per_seq, uint64_t *anc_out, int32_t *seq_tile_start, int32_t *seq_ntiles,
                     int32_t *seq_npages, int32_t *status, int32_t *error_flag, __nv_bfloat16 *out, float *lse,
                     int Hq, int D, cudaStream_t st) {
-    prepare_kernel<<<1, 1024, 0, st>>>(padded, c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages, parent, B, T,
-                                       n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles,
-                                       seq_npages, status, error_flag, out, lse, Hq, D);
+    launch_pdl(prepare_kernel, dim3(1), dim3(1024), 0, st, padded, c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages,
+               parent, B, T, n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles, seq_npages, status,
+               error_flag, out, lse, Hq, D);
 }
 
 }  // namespace reader

@@ -438,6 +438,66 @@ def test_commit_page_crossing_capacity_and_prefix_guard(rd):
         np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
 
 
+def fused_accept_commit(rd, w, logits=True, target_ids=None, update=True):
+    from paper_2508_09072_b200 import binding
+    d = binding.to_device(w, with_logits=logits)
+    tgt = None if target_ids is None else torch.from_numpy(target_ids).cuda()
+    r = rd.accept_commit(d.parent, d.node_tokens, w.max_path, d.cache, d.k_tree, d.v_tree,
+                         logits=d.logits if logits else None, target_ids=tgt, update_seq_lens=update)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in r.items()}
+    got.update(k_pool=binding.bf16_bits(d.cache.k_pool), v_pool=binding.bf16_bits(d.cache.v_pool),
+               seq_lens=d.cache.seq_lens.cpu().numpy())
+    return got
+
+
+def check_fused(w, got, target, update=True):
+    a = oracle.accept(w.parent, w.node_tokens, target, w.max_path)
+    c = oracle.kv_commit(w.k_pool, w.v_pool, w.page_table, w.seq_lens, w.shared_prefix_len, w.k_tree, w.v_tree,
+                         a["path"], a["n_acc"], update_seq_lens=update)
+    np.testing.assert_array_equal(got["target_ids"], target)
+    for k in ("path", "n_acc", "bonus", "status"):
+        np.testing.assert_array_equal(got[k], a[k], err_msg=k)
+    for k in ("k_pool", "v_pool", "seq_lens", "slots"):
+        np.testing.assert_array_equal(got[k], c[k], err_msg=k)
+    np.testing.assert_array_equal(got["commit_status"], c["status"])
+
+
+@pytest.mark.parametrize("name", W.WORKLOADS)
+def test_accept_and_commit_in_one_launch_named_workloads(rd, name):
+    """reader_accept_commit against the oracle's acceptance followed by the oracle's commit."""
+    w = W.make(name, reduced=(name != "c1"))
+    for update in (True, False):
+        check_fused(w, fused_accept_commit(rd, w, update=update), oracle.argmax(w.logits), update)
+
+
+def test_accept_and_commit_in_one_launch_edge_cases(rd):
+    # given target ids instead of logits; a malformed tree; a sequence without room; a full-depth chain
+    T = 20
+    w = W.build_workload("s", 41, [60, 127, 200, 128 + 5, 64], T, 8, 4, 64, lambda r: W.chain_tree(T), max_path=16, vocab=16,
+                         shuffle_pages=True, with_logits=False, spare_pages=2)
+    rng = np.random.default_rng(42)
+    target = rng.integers(0, 16, size=(5, T)).astype(np.int32)
+    for j in range(1, T):                         # sequence 0 and 4 accept the whole chain (up to max_path)
+        w.node_tokens[0, j] = target[0, j - 1]
+        w.node_tokens[4, j] = target[4, j - 1]
+    w.node_tokens[3, 1:4] = target[3, 0:3]      # sequence 3 accepts four nodes at least
+    w.node_tokens[3, 4] = (target[3, 3] + 1) % 16
+    w.parent[2, 7] = 9                            # sequence 2: a parent after its child
+    w.page_table[1, 2:] = -1                      # sequence 1: no page for positions >= 128
+    w.node_tokens[1, 1:3] = target[1, 0:2]
+    w.shared_prefix_len = 0
+    got = fused_accept_commit(rd, w, logits=False, target_ids=target)
+    check_fused(w, got, target)
+    assert got["status"].tolist()[2] == oracle.BAD_TREE and got["n_acc"].tolist()[0] == 16
+    assert got["commit_status"].tolist()[1] == oracle.CAPACITY
+
+
+def test_accept_and_commit_in_one_launch_full_size_c3(rd):
+    w = W.make("c3")
+    check_fused(w, fused_accept_commit(rd, w), oracle.argmax(w.logits))
+
+
 # ------------------------------------------------------------------------------------ whole step
 def test_whole_step_then_next_step_sees_committed_rows(rd):
     """encode -> attention -> accept -> commit on the device, then a second attention call must
