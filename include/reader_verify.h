@@ -33,6 +33,9 @@
  *     outside the pool, a length beyond the page table.  A sequence with a non-zero status gets
  *     defined outputs (attention rows and lse zero; n_acc 0, path -1, bonus -1; nothing
  *     committed) and does not disturb the others.  No kernel traps, asserts or waits unbounded.
+ *   - A context is bound to one device and is not thread-safe: it caches the TMA descriptors of the
+ *     tensors it saw last, so calls on one context come from one host thread at a time (use one
+ *     context per thread or serialise).  Calls on different contexts are independent.
  *   - An empty batch (batch = 0) is legal everywhere: the call returns READER_OK, launches nothing
  *     and looks at no tensor pointer.
  *   - Tree convention: node 0 is the root = the last token already chosen by the target model
