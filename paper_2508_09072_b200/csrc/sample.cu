@@ -158,9 +158,20 @@ __global__ void __launch_bounds__(kSampleThreads, 4) sample_kernel(const float *
                 __syncthreads();
                 const unsigned prefix = sh.sel_prefix;          // the digits above this one, already fixed
                 auto add = [&](unsigned key) {
-                    if (key >= floor_key && (pass == 0 || (key >> (shift + width)) == prefix))
-                        atomicAdd(&sh.hist[(key >> shift) & (nbins - 1)],
-                                  weighted ? sample_weight(sample_unkey(key), m, c) : 1ull);
+                    if (key >= floor_key && (pass == 0 || (key >> (shift + width)) == prefix)) {
+                        // a 64-bit sum kept by two 32-bit additions (low word first, its carry into the high
+                        // word): exact, and native 32-bit shared-memory atomics instead of a 64-bit one
+                        unsigned *bin = reinterpret_cast<unsigned *>(&sh.hist[(key >> shift) & (nbins - 1)]);
+                        if (!weighted) {
+                            atomicAdd(bin, 1u);                         // at most 2^21 keys: no carry
+                        } else {
+                            const unsigned long long wgt = sample_weight(sample_unkey(key), m, c);
+                            const unsigned lo = (unsigned)wgt, hi = (unsigned)(wgt >> 32);
+                            unsigned carry = 0;
+                            if (lo) carry = atomicAdd(bin, lo) > ~lo ? 1u : 0u;   // old + lo wrapped
+                            if (hi | carry) atomicAdd(bin + 1, hi + carry);
+                        }
+                    }
                 };
                 if (from_list) {
                     for (unsigned i = tid; i < sh.n_cand; i += kSampleThreads) add(sh.cand[i]);
