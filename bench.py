@@ -360,8 +360,9 @@ def run_ours(args):
 
         def model_step():
             d.cache.seq_lens.copy_(seq_lens0)
+            rd.verify_prepare(m_caches[0], d.parent, w.n_q_heads, status=status, workspace=ws)   # once for all layers
             for c in m_caches:
-                rd.verify_attn(d.q, d.k_tree, d.v_tree, c, d.parent, w.scale, out=out, status=status, workspace=ws)
+                rd.verify_attn_prepared(d.q, d.k_tree, d.v_tree, c, d.parent, w.scale, ws, out=out)
             rd.accept(d.parent, d.node_tokens, w.max_path, logits=d.logits, target_ids=tgt, workspace=ws, outs=acc_out)
             rd.kv_commit_layers(m_caches, lk[:Lm], lv[:Lm], acc_out[0], acc_out[1], slots=slots, status=cstat)
 
@@ -397,7 +398,7 @@ def run_ours(args):
         model_step_res = {"layers": Lm, "ms_per_step": {"call_by_call": t_model_eager, "cuda_graph": t_model_graph},
                           "tokens_per_s": B * T / (t_model_graph * 1e-3), "algorithmic_bytes": kv_bytes,
                           "gbs": kv_bytes / (t_model_graph * 1e-3) / 1e9,
-                          "note": "every layer's verify attention on its own cache + one acceptance + one commit into all layers; "
+                          "note": "checks and work partition once, every layer's verify attention on its own cache, one acceptance, one commit into all layers; "
                                   "not the metric's step (one layer), reported beside it"}
         del m_caches, mgraph
     except Exception as exc:                                  # reported, never hidden

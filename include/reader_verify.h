@@ -13,7 +13,8 @@
  *     reader_accept        target argmax + longest consistent root path          (Algorithm 5)
  *     reader_kv_commit     accepted K/V rows -> cache tail, seq_lens += n_acc    (Algorithm 4)
  *   and, beside these: reader_sample_targets (the sampling policies of Appendix C in place of the
- *   argmax), reader_accept_commit (acceptance and commit in one launch), reader_kv_commit_layers (all
+ *   argmax), reader_verify_prepare / reader_verify_attn_prepared (the per-step part of the attention call
+ *   done once for all layers), reader_accept_commit (acceptance and commit in one launch), reader_kv_commit_layers (all
  *   layers of a model in one launch), reader_kv_rearrange
  *   (Algorithm 4 on the paper's padded cache layout), reader_verify_attn_padded /
  *   reader_padded_append / reader_padded_rearrange (the padded cache of Sec. 4.3 run as a cache, to be
@@ -263,6 +264,32 @@ reader_status reader_kv_commit_layers(reader_ctx *ctx, const reader_kv_cache *ca
 reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t batch, int32_t n_kv_heads,
                                   int32_t capacity, int32_t head_dim, uint8_t *valid, int32_t *lengths_out,
                                   void *stream);
+
+/*
+ * reader_verify_attn in two parts, for a model with several layers: all layers of a step see the same
+ * trees, lengths and block table, so the checks, the masks and the work partition are made once
+ * (reader_verify_prepare) and every layer then runs only its attention and combine kernels
+ * (reader_verify_attn_prepared) -- one launch and several microseconds fewer per layer.
+ *
+ * reader_verify_prepare: cache->page_table / seq_lens / shapes and tree are read (k_pool, v_pool are
+ * not); status_out (i32 [batch]) receives the status words of reader_verify_attn and stays in use by
+ * the prepared calls.  The result lives in `workspace`.
+ * reader_verify_attn_prepared: same arguments as reader_verify_attn, with this layer's q, k_tree,
+ * v_tree, pools and out; workspace, batch, tree (parent and anc_mask pointers), n_q_heads and the
+ * cache's page_table, seq_lens and shapes must be the ones given to the last reader_verify_prepare on
+ * this context, else READER_ERR_INVALID_ARG.  Between the two nothing may change seq_lens, the page
+ * table or the trees, and no other reader_verify_attn* call may use the workspace (reader_accept* may).
+ * Rows of a rejected sequence are zeroed in every layer's out.  A bounded wait that gives up in one
+ * layer marks all later layers of the step as well (READER_ERR_TIMEOUT in status_out, zero rows).
+ */
+reader_status reader_verify_prepare(reader_ctx *ctx, const reader_kv_cache *cache, const reader_tree *tree,
+                                    int32_t n_q_heads, void *workspace, size_t workspace_bytes,
+                                    int32_t *status_out, void *stream);
+reader_status reader_verify_attn_prepared(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
+                                          const void *v_tree, const reader_kv_cache *cache,
+                                          const reader_tree *tree, float softmax_scale, void *out,
+                                          float *lse_out, void *workspace, size_t workspace_bytes,
+                                          void *stream);
 
 /*
  * The padded batch cache of Sec. 4.3 as a cache in its own right: the layout the paper starts from,

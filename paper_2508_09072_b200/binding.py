@@ -26,7 +26,8 @@ EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_se
            "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
            "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers",
-           "reader_accept_commit", "reader_padded_workspace_bytes", "reader_verify_attn_padded", "reader_padded_append", "reader_padded_rearrange")
+           "reader_accept_commit", "reader_verify_prepare", "reader_verify_attn_prepared",
+           "reader_padded_workspace_bytes", "reader_verify_attn_padded", "reader_padded_append", "reader_padded_rearrange")
 
 
 class ReaderError(RuntimeError):
@@ -97,6 +98,12 @@ def load_library() -> ctypes.CDLL:
     lib.reader_kv_rearrange.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p,
                                         c_void_p, c_void_p]
     lib.reader_kv_rearrange.restype = c_int32
+    lib.reader_verify_prepare.argtypes = [c_void_p, POINTER(_KvCache), POINTER(_Tree), c_int32, c_void_p, c_size_t, c_void_p,
+                                          c_void_p]
+    lib.reader_verify_prepare.restype = c_int32
+    lib.reader_verify_attn_prepared.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, POINTER(_KvCache),
+                                                POINTER(_Tree), c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.reader_verify_attn_prepared.restype = c_int32
     lib.reader_accept_commit.argtypes = [c_void_p, POINTER(_Tree), c_void_p, c_void_p, c_int32, c_void_p, c_int32,
                                          POINTER(_KvCache), c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p,
                                          c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p]
@@ -267,6 +274,40 @@ class Reader:
         if st != OK:
             raise ReaderError(st, "reader_verify_attn")
         return out, status
+
+    def verify_prepare(self, cache: KvCache, parent: torch.Tensor, n_q_heads: int, anc_mask: Optional[torch.Tensor] = None,
+                       status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+        """reader_verify_prepare: the per-step part of verify_attn (checks, masks, work partition), once for
+        all layers.  Returns (status, workspace); pass both tensors' owners on to verify_attn_prepared."""
+        _dev(parent, torch.int32, "parent")
+        B, T = parent.shape
+        c = cache._c()
+        status = status if status is not None else torch.empty(B, dtype=torch.int32, device=parent.device)
+        ws = workspace if workspace is not None else self.workspace(max(B, 1), T, n_q_heads, c.n_kv_heads, c.head_dim)
+        tree = _Tree(B, T, parent.data_ptr(), None if anc_mask is None else anc_mask.data_ptr())
+        st = self.lib.reader_verify_prepare(self._h, ctypes.byref(c), ctypes.byref(tree), int(n_q_heads), _ptr(ws), ws.numel(),
+                                            _ptr(status), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_verify_prepare")
+        return status, ws
+
+    def verify_attn_prepared(self, q: torch.Tensor, k_tree: torch.Tensor, v_tree: torch.Tensor, cache: KvCache,
+                             parent: torch.Tensor, scale: float, workspace: torch.Tensor,
+                             anc_mask: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                             lse: Optional[torch.Tensor] = None):
+        """reader_verify_attn_prepared: one layer's attention and combine on the schedule verify_prepare left
+        in `workspace`."""
+        _dev(q, torch.bfloat16, "q"); _dev(k_tree, torch.bfloat16, "k_tree"); _dev(v_tree, torch.bfloat16, "v_tree")
+        B, T, Hq, D = q.shape
+        out = out if out is not None else torch.empty_like(q)
+        tree = _Tree(B, T, parent.data_ptr(), None if anc_mask is None else anc_mask.data_ptr())
+        c = cache._c()
+        st = self.lib.reader_verify_attn_prepared(self._h, _ptr(q), Hq, _ptr(k_tree), _ptr(v_tree), ctypes.byref(c),
+                                                  ctypes.byref(tree), float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                                  workspace.numel(), _stream())
+        if st != OK:
+            raise ReaderError(st, "reader_verify_attn_prepared")
+        return out
 
     def verify_attn_padded(self, q: torch.Tensor, k_tree: torch.Tensor, v_tree: torch.Tensor, cache: PaddedCache,
                            parent: torch.Tensor, scale: float, anc_mask: Optional[torch.Tensor] = None,

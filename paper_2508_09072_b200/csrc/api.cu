@@ -85,6 +85,7 @@ reader_status reader_create(reader_ctx **out, int device) {
     ctx->attn_kernel = 0;
     ctx->ev_start = ctx->ev_stop = nullptr;
     ctx->ev_acc_start = ctx->ev_acc_stop = nullptr;
+    ctx->prepared = PreparedRecord{};
     reader_status st = sm100_host_init(&ctx->sm100, device);
     if (st != READER_OK) {
         delete ctx;
@@ -160,9 +161,11 @@ namespace {
 // workspace is carved, the parameter block completed and the three kernels are enqueued.
 // `p` arrives with the cache fields set; `bits_offset` is where the packed mask of a padded cache
 // lives in the workspace (unused for the paged cache).
+enum AttnMode { kPrepareAndRun, kPrepareOnly, kRunPrepared };
+
 reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cache *paged, const reader_padded_cache *padded,
                               const reader_tree *tree, float softmax_scale, void *workspace, size_t workspace_bytes,
-                              void *stream) {
+                              void *stream, AttnMode mode = kPrepareAndRun) {
     const int B = p.B, T = p.T, Hkv = p.Hkv, D = p.D;
     const int n_mtiles = (T * p.G + kTileM - 1) / kTileM;
     const int n_tree_tiles = (T + kPage - 1) / kPage;
@@ -202,14 +205,16 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     }
 
     const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
-    if (ctx->attn_kernel == 2 && !tc_ok) return READER_ERR_UNSUPPORTED;
+    if (ctx->attn_kernel == 2 && !tc_ok && mode != kPrepareOnly) return READER_ERR_UNSUPPORTED;
     const bool use_tc = tc_ok && ctx->attn_kernel != 1;
     p.sched.n_ctas = max_ctas(ctx);   // two resident CTAs per SM for both kernels
 
-    launch_prepare(paged ? *paged : none, pin, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
+    if (mode != kRunPrepared)
+        launch_prepare(paged ? *paged : none, pin, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
                    tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
                    reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
                    reinterpret_cast<int32_t *>(ws + w.seq_npages), p.status, p.error_flag, p.out, p.lse, p.Hq, D, st);
+    if (mode == kPrepareOnly) return launch_status();
     if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
     if (use_tc) {
         if (reader_status s = launch_attn_sm100(&ctx->sm100, p, st)) return s;
@@ -261,6 +266,77 @@ reader_status reader_verify_attn(reader_ctx *ctx, const void *q, int32_t n_q_hea
     p.pool_rows = (int64_t)cache->num_pages * Hkv * kPage;
     p.shared_prefix_pages = cache->shared_prefix_len / kPage;
     return run_verify_attn(ctx, p, cache, nullptr, tree, softmax_scale, workspace, workspace_bytes, stream);
+}
+
+reader_status reader_verify_prepare(reader_ctx *ctx, const reader_kv_cache *cache, const reader_tree *tree,
+                                    int32_t n_q_heads, void *workspace, size_t workspace_bytes, int32_t *status_out,
+                                    void *stream) {
+    if (!ctx || !cache || !tree) return READER_ERR_INVALID_ARG;
+    ctx->prepared.valid = false;
+    if (tree->batch == 0) return READER_OK;
+    if (!workspace || !status_out || !cache->page_table || !cache->seq_lens || !tree->parent) return READER_ERR_INVALID_ARG;
+    const int B = tree->batch, T = tree->n_nodes, Hq = n_q_heads, Hkv = cache->n_kv_heads, D = cache->head_dim;
+    if (B < 0 || T < 1 || T > kMaxNodes || Hq < 1 || Hkv < 1 || cache->num_pages < 0 || cache->max_pages_per_seq < 1)
+        return READER_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128) || cache->page_size != kPage) return READER_ERR_UNSUPPORTED;
+    if (cache->shared_prefix_len < 0 || cache->shared_prefix_len % kPage != 0) return READER_ERR_INVALID_ARG;
+    if (!aligned16(tree->anc_mask) || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return READER_ERR_INVALID_ARG;
+    AttnParams p{};
+    p.page_table = cache->page_table;
+    p.seq_lens = cache->seq_lens;
+    p.status = status_out;
+    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
+    p.max_pages = cache->max_pages_per_seq;
+    p.num_pages = cache->num_pages;
+    p.pool_rows = (int64_t)cache->num_pages * Hkv * kPage;
+    p.shared_prefix_pages = cache->shared_prefix_len / kPage;
+    const reader_status s = run_verify_attn(ctx, p, cache, nullptr, tree, 1.0f, workspace, workspace_bytes, stream, kPrepareOnly);
+    if (s != READER_OK) return s;
+    PreparedRecord &r = ctx->prepared;
+    r.valid = true;
+    r.workspace = workspace; r.page_table = cache->page_table; r.seq_lens = cache->seq_lens;
+    r.parent = tree->parent; r.anc_mask = tree->anc_mask; r.status = status_out;
+    r.B = B; r.T = T; r.Hq = Hq; r.Hkv = Hkv; r.D = D;
+    r.max_pages = cache->max_pages_per_seq; r.num_pages = cache->num_pages; r.shared_prefix_len = cache->shared_prefix_len;
+    return READER_OK;
+}
+
+reader_status reader_verify_attn_prepared(reader_ctx *ctx, const void *q, int32_t n_q_heads, const void *k_tree,
+                                          const void *v_tree, const reader_kv_cache *cache, const reader_tree *tree,
+                                          float softmax_scale, void *out, float *lse_out, void *workspace,
+                                          size_t workspace_bytes, void *stream) {
+    if (!ctx || !cache || !tree) return READER_ERR_INVALID_ARG;
+    if (tree->batch == 0) return READER_OK;
+    if (!q || !k_tree || !v_tree || !out || !workspace || !cache->k_pool || !cache->v_pool) return READER_ERR_INVALID_ARG;
+    const PreparedRecord &r = ctx->prepared;
+    const int B = tree->batch, T = tree->n_nodes, Hq = n_q_heads, Hkv = cache->n_kv_heads, D = cache->head_dim;
+    // the schedule in the workspace was made for one problem: same workspace, batch, tree and block table only
+    if (!r.valid || r.workspace != workspace || r.B != B || r.T != T || r.Hq != Hq || r.Hkv != Hkv || r.D != D ||
+        r.page_table != cache->page_table || r.seq_lens != cache->seq_lens || r.max_pages != cache->max_pages_per_seq ||
+        r.num_pages != cache->num_pages || r.shared_prefix_len != cache->shared_prefix_len || r.parent != tree->parent ||
+        r.anc_mask != tree->anc_mask || cache->page_size != kPage || !(softmax_scale == softmax_scale))
+        return READER_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(cache->k_pool) || !aligned16(cache->v_pool) ||
+        !aligned16(out))
+        return READER_ERR_INVALID_ARG;
+    AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.k_tree = static_cast<const __nv_bfloat16 *>(k_tree);
+    p.v_tree = static_cast<const __nv_bfloat16 *>(v_tree);
+    p.k_pool = static_cast<const __nv_bfloat16 *>(cache->k_pool);
+    p.v_pool = static_cast<const __nv_bfloat16 *>(cache->v_pool);
+    p.page_table = cache->page_table;
+    p.seq_lens = cache->seq_lens;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse_out;
+    p.status = r.status;
+    p.zero_rejected = 1;
+    p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
+    p.max_pages = cache->max_pages_per_seq;
+    p.num_pages = cache->num_pages;
+    p.pool_rows = (int64_t)cache->num_pages * Hkv * kPage;
+    p.shared_prefix_pages = cache->shared_prefix_len / kPage;
+    return run_verify_attn(ctx, p, cache, nullptr, tree, softmax_scale, workspace, workspace_bytes, stream, kRunPrepared);
 }
 
 size_t reader_padded_workspace_bytes(const reader_ctx *ctx, int32_t max_batch, int32_t max_nodes, int32_t n_q_heads,

@@ -36,6 +36,16 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
         for (size_t i = me; i < (size_t)p.B; i += nthreads) p.status[i] = err;
         return;
     }
+    if (p.zero_rejected) {   // block-uniform loop: every block takes some of the sequences
+        const int nblocks = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
+        for (int b = me; b < p.B; b += nblocks) {
+            if (p.status[b] == READER_OK) continue;
+            uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)b * p.T * p.Hq * D);
+            for (size_t i = threadIdx.x; i < (size_t)p.T * p.Hq * D / 8; i += blockDim.x) o[i] = make_uint4(0, 0, 0, 0);
+            if (p.lse)
+                for (int i = threadIdx.x; i < p.T * p.Hq; i += blockDim.x) p.lse[(size_t)b * p.T * p.Hq + i] = 0.f;
+        }
+    }
     if (d.b < 0) return;
     const int rows = min(kTileM, p.T * p.G - d.mt * kTileM);
     const bool has_cols = lane * 4 < D;

@@ -192,6 +192,8 @@ struct AttnParams {
     // whether row t * kPage + r of sample b is a real entry (0 at and beyond the common extent).
     const uint64_t *valid_bits;
     int bits_per_seq, cap;
+    int zero_rejected;         // the combine kernel zeroes the rows of sequences whose status word is set (the
+                               // preparation ran in an earlier call and could not know this call's output)
     Sched sched;
 };
 

@@ -121,7 +121,8 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
             seq_ntiles[b] = st == READER_OK ? npages + n_tree_tiles : 0;
             seq_npages[b] = st == READER_OK ? npages : 0;
         }
-        if (st != READER_OK) {   // a rejected sequence gets defined output: zero rows, zero lse
+        if (st != READER_OK && out) {   // a rejected sequence gets defined output: zero rows, zero lse
+                                         // (out == nullptr: the attention calls that follow do it per layer)
             const size_t n16 = (size_t)T * Hq * D / 8;
             uint4 *o = reinterpret_cast<uint4 *>(out + (size_t)b * T * Hq * D);
             for (size_t i = lane; i < n16; i += 32) o[i] = make_uint4(0, 0, 0, 0);

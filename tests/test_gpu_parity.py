@@ -626,6 +626,66 @@ def test_multi_layer_step_in_one_graph_matches_oracle_layer_by_layer(rd):
         np.testing.assert_array_equal(slots.cpu().numpy(), com["slots"])
 
 
+@pytest.mark.parametrize("kernel", [1, 2])
+def test_prepare_once_then_every_layer(rd, kernel):
+    """reader_verify_prepare + reader_verify_attn_prepared per layer against the oracle, one rejected
+    sequence included: its rows must be zero in every layer's output."""
+    from paper_2508_09072_b200 import binding
+    n_layers = 3
+    w = W.make("c3", reduced=True)
+    w.parent[1, 9] = 12                                  # sequence 1: a parent after its child
+    rng = np.random.default_rng(91)
+    layers = [(w.q, w.k_tree, w.v_tree, w.k_pool, w.v_pool)]
+    for _ in range(n_layers - 1):
+        layers.append(tuple(W.normal_bf16(rng, a.shape) for a in layers[0]))
+    d = binding.to_device(w, with_logits=False)
+    dev = [tuple(binding.bf16_tensor(a, "cuda") for a in lay) for lay in layers]
+    caches = [binding.KvCache(l[3], l[4], d.cache.page_table, d.cache.seq_lens, 0) for l in dev]
+    ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    ws.fill_(0xFF)
+    rd.set_attn_kernel(kernel)
+    try:
+        status, _ = rd.verify_prepare(caches[0], d.parent, w.n_q_heads, workspace=ws)
+        outs, lses = [], []
+        for l in range(n_layers):
+            out = torch.full_like(d.q, 3.0)
+            lse = torch.full((w.batch, w.n_nodes, w.n_q_heads), 7.0, dtype=torch.float32, device="cuda")
+            rd.verify_attn_prepared(dev[l][0], dev[l][1], dev[l][2], caches[l], d.parent, w.scale, ws, out=out, lse=lse)
+            outs.append(out); lses.append(lse)
+        torch.cuda.synchronize()
+    finally:
+        rd.set_attn_kernel(0)
+    assert status.cpu().numpy().tolist() == [0, oracle.BAD_TREE, 0]
+    for l, (q, kt, vt, kp, vp) in enumerate(layers):
+        w_l = copy.copy(w)
+        w_l.q, w_l.k_tree, w_l.v_tree, w_l.k_pool, w_l.v_pool = q, kt, vt, kp, vp
+        got = W.bf16_bits_to_f32(binding.bf16_bits(outs[l])).astype(np.float64)
+        check_attn(w_l, got, status.cpu().numpy(), lses[l].cpu().numpy().astype(np.float64))
+        assert not got[1].any() and not lses[l][1].any().item()
+
+
+def test_prepared_call_refuses_another_problem(rd):
+    from paper_2508_09072_b200 import binding
+    w = W.make("c3", reduced=True)
+    d = binding.to_device(w, with_logits=False)
+    ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    other_ws = torch.empty_like(ws)
+    with pytest.raises(binding.ReaderError) as e:          # nothing prepared in that workspace
+        rd.verify_attn_prepared(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, other_ws)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    rd.verify_prepare(d.cache, d.parent, w.n_q_heads, workspace=ws)
+    rd.verify_attn_prepared(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, ws)
+    other_parent = d.parent.clone()
+    for args in ((d.q, d.k_tree, d.v_tree, d.cache, other_parent, w.scale, ws),                      # another tree tensor
+                 (d.q[:2], d.k_tree[:2], d.v_tree[:2], d.cache, d.parent, w.scale, ws),              # another batch
+                 (d.q, d.k_tree, d.v_tree, binding.KvCache(d.cache.k_pool, d.cache.v_pool, d.cache.page_table,
+                                                           d.cache.seq_lens.clone(), 0), d.parent, w.scale, ws)):
+        with pytest.raises(binding.ReaderError) as e:
+            rd.verify_attn_prepared(*args)
+        assert e.value.code == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+
+
 def test_thousands_of_calls_never_hit_a_bounded_wait(rd):
     """Every device-side wait is bounded, so a lost wake-up shows as READER_ERR_TIMEOUT in the status
     words of one call in many (and as a one-second stall) rather than as a hang.  The status maximum
