@@ -49,9 +49,12 @@
  * dominant key -> that V); probabilities sum to one; split-and-merge algebra;
  * sibling-order and page-permutation invariance; exhaustive acceptance on
  * all trees with <= 6 nodes against an independently written accepted-set
- * propagation; Eq. 1 statistics; the deterministic-losslessness loop.
- * Absolute attention values on random inputs beyond those pins: parity
- * unpinned (the paper prints no worked numeric example).
+ * propagation; Eq. 1 statistics; the deterministic-losslessness loop;
+ * random trees and random inputs against torch's attention under a mask
+ * derived by transitive closure (to 1e-12).  Every function in this file
+ * has at least one pin against something other than itself; none is
+ * "parity unpinned".  (The paper prints no worked numeric example, so no
+ * pin is a value quoted from it except the Eq. 1 table.)
  *
  * Layouts (row-major, last index fastest):
  *   q, out        [B][T][Hq][D]        k_tree, v_tree  [B][T][Hkv][D]
