@@ -117,12 +117,12 @@ const char *reader_status_string(reader_status s);
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
 
 /* Profiling aid (host call): when both are non-NULL cudaEvent_t handles, the next calls of
- * reader_verify_attn record `start` on the stream right before the main attention kernel and
+ * reader_verify_attn (and of its prepared and padded forms) record `start` on the stream right before the main attention kernel and
  * `stop` right after it (the preparation and combine kernels lie outside).  NULL, NULL turns it off. */
 reader_status reader_set_timing_events(reader_ctx *ctx, void *start, void *stop);
 
-/* The same for reader_accept called with logits: the events bracket the argmax kernel (the acceptance
- * walk that follows lies outside).  NULL, NULL turns it off. */
+/* The same for reader_accept and reader_accept_commit called with logits: the events bracket the argmax
+ * kernel (the acceptance walk that follows lies outside).  NULL, NULL turns it off. */
 reader_status reader_set_accept_timing_events(reader_ctx *ctx, void *start, void *stop);
 
 /* Bytes of device scratch that reader_verify_attn / reader_accept need for at most `max_batch`
