@@ -207,7 +207,15 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
     if (ctx->attn_kernel == 2 && !tc_ok && mode != kPrepareOnly) return READER_ERR_UNSUPPORTED;
     const bool use_tc = tc_ok && ctx->attn_kernel != 1;
-    p.sched.n_ctas = max_ctas(ctx);   // two resident CTAs per SM for both kernels
+    // Two resident CTAs per SM for both kernels -- fewer when the page table is too narrow to give that many
+    // CTAs work: on the device effective_ctas() never uses more than ceil(W / kMinTilesPerCta) lanes, and W
+    // cannot exceed the bound below, so the partition is the same and the launches are smaller.
+    {
+        const int64_t w_bound = (int64_t)B * Hkv * (max_pages + n_tree_tiles + kUnitOverhead);
+        const int64_t lanes = (w_bound + kMinTilesPerCta - 1) / kMinTilesPerCta;
+        const int64_t busy = (lanes < 1 ? 1 : lanes) * n_mtiles;
+        p.sched.n_ctas = (int)(busy < max_ctas(ctx) ? busy : max_ctas(ctx));
+    }
 
     if (mode != kRunPrepared)
         launch_prepare(paged ? *paged : none, pin, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
