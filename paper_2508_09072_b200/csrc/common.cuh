@@ -43,6 +43,7 @@ struct Segment {
     int span;                  // entries of the flat list this segment covers (overhead entries included)
     int unit_w0;               // flat index of the unit's first entry
     int ntiles, npages;
+    int len;                   // committed length of the sequence (segment_at_warp only; 0 with a padded cache)
     bool full;                 // covers the whole unit
     int slot;                  // partial slot when !full
 };
@@ -97,22 +98,53 @@ __device__ __forceinline__ Segment segment_at(const Sched &s, int B, int cta, in
     return g;
 }
 
-// Same result as segment_at, for a whole warp calling together: the sequence is found with one
-// round of parallel loads per 32 sequences instead of a chain of dependent ones.
-__device__ __forceinline__ Segment segment_at_warp(const Sched &s, int B, int cta, int w, int range_end, int lane) {
-    int b = 0;
-    for (int base = 0; base < B; base += 32) {
-        const int i = base + lane;
-        const unsigned le = __ballot_sync(0xffffffffu, i < B && s.seq_tile_start[i] <= w);
-        if (le) b = base + 31 - __clz(le);   // the starts never decrease: the set bits are a prefix
-        if (le != 0xffffffffu) break;
+// The schedule of up to 32 sequences held one sequence per lane: loaded once per warp with all loads in
+// flight together, so that finding a segment later costs shuffles instead of a chain of dependent global
+// loads (four round trips to L2 before a CTA's first tile could be requested).  With more than 32
+// sequences it stays empty and the lookups go to memory.
+struct WarpSched {
+    int start, ntiles, npages, len;
+};
+__device__ __forceinline__ WarpSched load_warp_sched(const Sched &s, const int32_t *seq_lens /*nullable*/, int B, int lane) {
+    WarpSched c{0x7fffffff, 0, 0, 0};
+    if (B <= 32 && lane < B) {
+        c.start = s.seq_tile_start[lane];
+        c.ntiles = s.seq_ntiles[lane];
+        c.npages = s.seq_npages[lane];
+        c.len = seq_lens ? seq_lens[lane] : 0;
     }
+    return c;
+}
+
+// Same result as segment_at (plus the sequence's committed length), for a whole warp calling together.
+__device__ __forceinline__ Segment segment_at_warp(const Sched &s, const WarpSched &c, const int32_t *seq_lens /*nullable*/,
+                                                   int B, int cta, int w, int range_end, int lane) {
     Segment g;
-    g.b = b;
-    g.ntiles = s.seq_ntiles[b];
-    g.npages = s.seq_npages[b];
+    int start_b;
+    if (B <= 32) {
+        const unsigned le = __ballot_sync(0xffffffffu, c.start <= w);   // the starts never decrease: a prefix of the lanes
+        const int b = le ? 31 - __clz(le) : 0;
+        g.b = b;
+        start_b = __shfl_sync(0xffffffffu, c.start, b);
+        g.ntiles = __shfl_sync(0xffffffffu, c.ntiles, b);
+        g.npages = __shfl_sync(0xffffffffu, c.npages, b);
+        g.len = __shfl_sync(0xffffffffu, c.len, b);
+    } else {
+        int b = 0;
+        for (int base = 0; base < B; base += 32) {   // one round of parallel loads per 32 sequences
+            const int i = base + lane;
+            const unsigned le = __ballot_sync(0xffffffffu, i < B && s.seq_tile_start[i] <= w);
+            if (le) b = base + 31 - __clz(le);
+            if (le != 0xffffffffu) break;
+        }
+        g.b = b;
+        start_b = s.seq_tile_start[b];
+        g.ntiles = s.seq_ntiles[b];
+        g.npages = s.seq_npages[b];
+        g.len = seq_lens ? seq_lens[b] : 0;
+    }
     const int per_unit = g.ntiles + kUnitOverhead;          // entries of one unit: overhead first, then its tiles
-    int local = w - s.seq_tile_start[b];
+    int local = w - start_b;
     int unit = local / per_unit;
     const int pos = local - unit * per_unit;
     const int pos_end = min(per_unit, pos + (range_end - w));

@@ -127,10 +127,6 @@ __device__ __forceinline__ bool ready(uint32_t bar, uint32_t parity) {
 // The cache kind is a compile-time choice (kPadded: the padded batch cache of Sec. 4.3, else the paged
 // cache), so that neither pays for the other's addressing.
 template <bool kPadded>
-__device__ __forceinline__ int len_of(const AttnParams &p, int b) {
-    if constexpr (kPadded) return 0; else return p.seq_lens[b];
-}
-template <bool kPadded>
 __device__ __forceinline__ uint64_t visible_of(const AttnParams &p, int b, int t, int L) {
     if constexpr (kPadded) {
         return p.valid_bits[(size_t)b * p.bits_per_seq + t];
@@ -158,26 +154,26 @@ struct TileCursor {
         if constexpr (kPadded) cache_page = 0;
         else cache_page = (tt < sg.tile_end && tt < sg.npages) ? p.page_table[(size_t)sg.b * p.max_pages + tt] : 0;
     }
-    __device__ __forceinline__ void next_segment(const AttnParams &p, int cta, int lane) {
+    __device__ __forceinline__ void next_segment(const AttnParams &p, const WarpSched &ws, int cta, int lane) {
         active = false;
         while (w < w_end) {   // segments without a real tile (a range that ends among overhead entries) are skipped
-            sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            sg = segment_at_warp(p.sched, ws, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
             w += sg.span;
             if (sg.tile_end > sg.tile_begin) { active = true; break; }
         }
         if (!active) return;
-        L = len_of<kPadded>(p, sg.b);
+        L = sg.len;
         t = sg.tile_begin;
         refill(p, lane);
     }
-    __device__ __forceinline__ void init(const AttnParams &p, int cta, int lane, int w_begin, int w_end_) {
+    __device__ __forceinline__ void init(const AttnParams &p, const WarpSched &ws, int cta, int lane, int w_begin, int w_end_) {
         w = w_begin; w_end = w_end_; it = 0;
-        next_segment(p, cta, lane);
+        next_segment(p, ws, cta, lane);
     }
     __device__ __forceinline__ int page() const { return __shfl_sync(0xffffffffu, cache_page, t - cache_t0); }
-    __device__ __forceinline__ void advance(const AttnParams &p, int cta, int lane) {
+    __device__ __forceinline__ void advance(const AttnParams &p, const WarpSched &ws, int cta, int lane) {
         ++t; ++it;
-        if (t == sg.tile_end) next_segment(p, cta, lane);
+        if (t == sg.tile_end) next_segment(p, ws, cta, lane);
         else if (t - cache_t0 == 32) refill(p, lane);
     }
 };
@@ -268,6 +264,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     // everything above overlapped the preparation kernel; its results are read from here on
     grid_dependency_wait();
     grid_launch_dependents();
+    const WarpSched wsched = load_warp_sched(p.sched, kPadded ? nullptr : p.seq_lens, p.B, lane);   // in flight with W
     const int W = p.sched.seq_tile_start[p.B];
     const CtaWork cw = cta_work(p.sched, cta, W);
     const int w_begin = cw.w_begin, w_end = cw.w_end;
@@ -286,8 +283,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         const uint64_t stream_policy = l2_policy_evict_first();
         const int first_streamed_tile = (p.sched.n_mtiles == 1 && p.shared_prefix_pages == 0) ? 0 : 0x7fffffff;
         TileCursor<kPadded> kc, vc;
-        kc.init(p, cta, lane, w_begin, w_end);
-        vc.init(p, cta, lane, w_begin, w_end);
+        kc.init(p, wsched, cta, lane, w_begin, w_end);
+        vc.init(p, wsched, cta, lane, w_begin, w_end);
         // the query tile of the next segment goes in as soon as the last score product of the
         // current one has retired (Q is single-buffered)
         int q_w = w_begin, q_seg = 0;
@@ -296,7 +293,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         while (kc.active || vc.active || q_w < w_end) {
             bool moved = false;
             if (q_w < w_end && ready(bar(&bars->q_empty), (q_seg & 1) ^ 1)) {
-                const Segment sg = segment_at_warp(p.sched, p.B, cta, q_w, w_end, lane);
+                const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, q_w, w_end, lane);
                 q_w += sg.span;
                 if (sg.tile_end <= sg.tile_begin) continue;   // no real tile: no query tile
                 if (lane == 0) {
@@ -315,7 +312,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStagesK) & 1) ^ 1)) {
                     load_tile<D, kPadded>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
-                    kc.advance(p, cta, lane);
+                    kc.advance(p, wsched, cta, lane);
                     moved = true;
                 }
             }
@@ -324,7 +321,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStagesV) & 1) ^ 1)) {
                     load_tile<D, kPadded>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
-                    vc.advance(p, cta, lane);
+                    vc.advance(p, wsched, cta, lane);
                     moved = true;
                 }
             }
@@ -352,7 +349,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int i = 0, seg = 0;
         int w = w_begin;
         while (w < w_end && !*abort_s) {
-            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += sg.span;
             if (n <= 0) continue;
@@ -386,11 +383,11 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int i = 0;
         int w = w_begin;
         while (w < w_end && !*abort_s) {
-            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += sg.span;
             if (n <= 0) continue;
-            const int L = len_of<kPadded>(p, sg.b);
+            const int L = sg.len;
             uint64_t vis_next = 0;
             if constexpr (kPadded) vis_next = sg.tile_begin < sg.npages ? visible_of<true>(p, sg.b, sg.tile_begin, L) : 0;
             for (int tl = 0; tl < n; ++tl, ++i) {
@@ -472,11 +469,11 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int w = w_begin;
         if (tid == 0) p.split_desc[cta].b = -1;
         while (w < w_end) {
-            const Segment sg = segment_at_warp(p.sched, p.B, cta, w, w_end, lane);
+            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
             if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
             w += sg.span;
             if (sg.tile_end <= sg.tile_begin) continue;
-            const int L = len_of<kPadded>(p, sg.b);
+            const int L = sg.len;
             const int grow = sg.mt * kTileM + tid;
             const bool row_ok = grow < p.T * p.G;
             const int j = row_ok ? grow / p.G : 0;
