@@ -686,6 +686,26 @@ def test_prepared_call_refuses_another_problem(rd):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("name", ["c2", "c3", "c5"])
+def test_repeated_calls_return_the_same_bits(rd, name):
+    """The work partition is static and partials are merged in a fixed order: the same inputs give the
+    same output bits on every call, through the plain call and through the prepared one."""
+    from paper_2508_09072_b200 import binding
+    w = W.make(name, reduced=True, with_logits=False)
+    d = binding.to_device(w, with_logits=False)
+    ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+    first, _ = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, workspace=ws)
+    first = first.clone()
+    for i in range(12):
+        if i % 2:
+            out, _ = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, workspace=ws)
+        else:
+            rd.verify_prepare(d.cache, d.parent, w.n_q_heads, workspace=ws)
+            out = rd.verify_attn_prepared(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, ws)
+        assert torch.equal(out, first)
+    torch.cuda.synchronize()
+
+
 def test_thousands_of_calls_never_hit_a_bounded_wait(rd):
     """Every device-side wait is bounded, so a lost wake-up shows as READER_ERR_TIMEOUT in the status
     words of one call in many (and as a one-second stall) rather than as a hang.  The status maximum
