@@ -160,6 +160,40 @@ def test_attn_random_shapes(rd):
             raise AssertionError(f"case {case}: T={T} G={G} Hkv={Hkv} D={D} lens={lens}: {e}")
 
 
+def test_attn_random_shapes_larger_batches_and_prepared_calls(rd):
+    """More seeded random shapes with up to 39 sequences (beyond the 32 a warp keeps the schedule of),
+    rotating through the automatic kernel choice, the tensor-core kernel alone and the prepared call."""
+    from paper_2508_09072_b200 import binding
+    rng = np.random.default_rng(777)
+    for case in range(36):
+        T = int(rng.choice([1, 2, 3, 7, 16, 31, 32, 33, 63, 64, 65, 100, 127, 128]))
+        G = int(rng.choice([1, 2, 4, 8, 16]))
+        Hkv = int(rng.choice([1, 2, 3, 8]))
+        D = int(rng.choice([64, 128]))
+        B = int(rng.integers(1, 40))
+        lens = [int(x) for x in rng.choice([0, 1, 5, 63, 64, 65, 127, 128, 129, 200, 333, 640, 1000], size=B)]
+        w = W.build_workload("r", 777000 + case, lens, T, G * Hkv, Hkv, D,
+                             lambda r: W.capped_recursive_tree(r, T, 12, 4) if T > 1 else np.array([-1], np.int32),
+                             max_path=12, vocab=16, shuffle_pages=True, with_logits=False, spare_pages=2)
+        mode = case % 3
+        if mode < 2:
+            got, status, lse = gpu_attn(rd, w, kernel=0 if mode == 0 else 2)
+        else:
+            d = binding.to_device(w, with_logits=False)
+            ws = rd.workspace(B, T, G * Hkv, Hkv, D)
+            ws.fill_(0xFF)
+            lse_t = torch.empty((B, T, G * Hkv), dtype=torch.float32, device="cuda")
+            st, _ = rd.verify_prepare(d.cache, d.parent, G * Hkv, workspace=ws)
+            out = rd.verify_attn_prepared(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, ws, lse=lse_t)
+            torch.cuda.synchronize()
+            got = W.bf16_bits_to_f32(binding.bf16_bits(out)).astype(np.float64)
+            status, lse = st.cpu().numpy(), lse_t.cpu().numpy().astype(np.float64)
+        try:
+            check_attn(w, got, status, lse)
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: T={T} G={G} Hkv={Hkv} D={D} B={B} lens={lens} mode={mode}: {e}")
+
+
 EXTREMES = [
     # B, T, G, Hkv, D, max committed length
     (300, 4, 2, 1, 64, 150),      # more sequences than CTAs
