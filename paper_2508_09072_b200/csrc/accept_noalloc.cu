@@ -80,6 +80,7 @@ extern "C" reader_status reader_accept_noalloc(reader_ctx *ctx, const reader_tre
 
     // enough blocks to fill the GPU, at least 2048 columns each, never more than the array holds
     int64_t splits = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;
+    if (splits < 3) splits = 3;   // as in reader_accept: never one block per row
     const int64_t by_width = vocab / 2048 > 0 ? vocab / 2048 : 1;
     if (splits > by_width) splits = by_width;
     if (splits > kSplitsCap) splits = kSplitsCap;
