@@ -30,7 +30,7 @@ UNIT = "tokens/s"
 LAUNCHES_PER_STEP = 5   # prepare, attention, combine, argmax, acceptance walk + commit
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised under
 # profiles/ (C3 only); None when the kernel has changed since its counters were taken.
-NCU_TRAFFIC = {("verify_attn", "c3"): 329.3e6, ("accept (target argmax)", "c3"): 528.5e6}
+NCU_TRAFFIC = {("verify_attn", "c3"): 329.3e6, ("accept (target argmax)", "c3"): 528.4e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

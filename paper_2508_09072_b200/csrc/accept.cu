@@ -22,12 +22,12 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ l
         const float4 *v4 = reinterpret_cast<const float4 *>(src + c0);
         const int n4 = (c1 - c0) >> 2;
         int i = threadIdx.x;
-        for (; i + 3 * 256 < n4; i += 4 * 256) {
-            float4 a[4];
+        for (; i + 7 * 256 < n4; i += 8 * 256) {
+            float4 a[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) a[u] = __ldcs(v4 + i + u * 256);
+            for (int u = 0; u < 8; ++u) a[u] = __ldcs(v4 + i + u * 256);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 const int at = c0 + 4 * (i + u * 256);
                 if (a[u].x > best.v) { best.v = a[u].x; best.i = at; }
                 if (a[u].y > best.v) { best.v = a[u].y; best.i = at + 1; }
