@@ -1,21 +1,30 @@
 #!/usr/bin/env python
-"""Benchmark of one batched tree-verification step (tree attention, acceptance, KV commit).
+"""Benchmark of the batched tree-verification attention (Sec. 3.2) and of the step around it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
 
-A step is one pass of the whole path over one synthetic batch: reader_verify_attn (ancestor masks
-encoded inside the call), reader_accept on the target logits, reader_kv_commit.  `value` is
-verified tree-tokens per second (batch * tree nodes / step time) with every input resident in
-HBM; `e2e` is the same with the step's inputs (Q, tree K/V, parent arrays, node tokens, logits)
-copied from pinned host memory and the results copied back inside the timed region.  Sequences are
-independent, so N GPUs run N replicas of the batch with no data-path collective (weak scaling).
-Prints one JSON line on rank 0.
+The headline is verify attention alone: `value` is verified tree-tokens per second of one
+reader_verify_attn call (batch * tree nodes / call time; ancestor masks encoded beforehand) with
+every input resident in HBM, and `roofline` is that call's attention kernel against the measured
+HBM copy bandwidth (or the measured bf16 tensor throughput where that binds).  A timed block is K
+calls; blocks are repeated until about a second has been timed and the median block is reported.
+`e2e` is the same call with the step's inputs (Q, tree K/V, parent arrays) copied from pinned host
+memory and the output copied back inside the timed region.  `workloads` holds the same
+measurement, L2 flushed before every call, for all five workloads C1..C5.  The acceptance (target
+argmax + walk) and the KV commit are timed separately (`kernels`), and the whole step
+(attention + acceptance + commit), a 32-layer model step and the side kernels are reported in
+keys of their own, never folded into the attention number.  Sequences are independent, so N GPUs
+run N replicas of the batch with no data-path collective (weak scaling).  Prints one JSON line on
+rank 0.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
+import re
 import subprocess
 import sys
 import threading
@@ -25,13 +34,16 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "verified tree-tokens/s (verify attention + acceptance + KV commit, 1 step)"
+METRIC = "verified tree-tokens/sec and achieved HBM GB/s (% of B200 peak), verify attn, 1 GPU"
 UNIT = "tokens/s"
-LAUNCHES_PER_STEP = 5   # prepare, attention, combine, argmax, acceptance walk + commit
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised under
-# profiles/ (C3 only); None when the kernel has changed since its counters were taken.
-NCU_TRAFFIC = {("verify_attn", "c3"): 329.3e6, ("accept (target argmax)", "c3"): 528.4e6}
+LAUNCHES_PER_ATTN_CALL = 3   # preparation, attention, combine
+LAUNCHES_PER_STEP = 5        # + argmax, acceptance walk with commit
+L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# ncu counters of one launch are kept as text under profiles/; each summary records the SHA-256 of the
+# kernel sources it was taken from, and a figure is used only while those sources are unchanged.
+TRAFFIC_PROFILES = {("verify_attn", "c3"): "attn_sm100_c3.md", ("argmax", "c3"): "argmax_c3.md"}
+TRAFFIC_SOURCES = {"verify_attn": ("verify_attn_sm100.cu", "common.cuh", "ptx_sm100.cuh"), "argmax": ("accept.cu",)}
 
 
 def load_peaks():
@@ -43,6 +55,33 @@ def load_peaks():
         except Exception:
             pass
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def source_digest(kind: str) -> str:
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES[kind]:
+        h.update(open(os.path.join(ROOT, "paper_2508_09072_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kind: str, workload: str):
+    """(bytes per launch, where from) out of the profile summary, or (None, why): the summary names the
+    digest of the sources its counters were taken from."""
+    name = TRAFFIC_PROFILES.get((kind, workload))
+    if not name:
+        return None, "no ncu capture of this workload"
+    try:
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+        m_b = re.search(r"^traffic-bytes-per-launch:\s*([0-9.eE+]+)", text, re.M)
+        m_s = re.search(r"^source-sha256-16:\s*([0-9a-f]{16})", text, re.M)
+        m_c = re.search(r"^captured-at-commit:\s*(\S+)", text, re.M)
+        if not (m_b and m_s):
+            return None, f"profiles/{name} states no counters"
+        if m_s.group(1) != source_digest(kind):
+            return None, f"kernel sources changed since the capture in profiles/{name}"
+        return float(m_b.group(1)), f"ncu capture in profiles/{name} (commit {m_c.group(1) if m_c else '?'}), not this run"
+    except OSError:
+        return None, f"profiles/{name} missing"
 
 
 class ClockSampler:
@@ -94,30 +133,56 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def fits_l2(w) -> bool:
+    return w.attn_algorithmic_bytes() <= 2 * L2_BYTES
+
+
 def workload_config(w, name):
     import numpy as np
     return {"workload": name, "batch": int(w.batch), "tree_nodes": int(w.n_nodes), "n_q_heads": int(w.n_q_heads),
             "n_kv_heads": int(w.n_kv_heads), "head_dim": int(w.head_dim), "page_size": int(w.page_size),
             "committed_tokens": int(np.sum(w.seq_lens)), "shared_prefix_len": int(w.shared_prefix_len),
-            "vocab": int(w.vocab), "l2": "no flush: per-step inputs exceed the 126 MB L2"
-            if w.attn_algorithmic_bytes() + w.logits_bytes() > 2 * 126e6 else "fits L2: numbers are warm-cache"}
+            "l2": ("L2 flushed before every call (a read pass over 512 MB): the call's inputs fit the 126 MB L2" if fits_l2(w)
+                   else "no flush: every call streams more K/V than the 126 MB L2 holds")}
+
+
+def median(xs):
+    xs = sorted(xs)
+    return xs[len(xs) // 2]
 
 
 # ------------------------------------------------------------------------------------------------
 # CPU baseline: the checker as it stands, on a bounded sample of the same workload
 # ------------------------------------------------------------------------------------------------
-def cpu_sample_step(w, seqs):
-    """Runs the CPU checker on the given sequences of the workload (whole step); returns seconds."""
+def one_sequence(w, b):
+    """Sequence b of the workload as a batch of one (views; the pool is shared)."""
     import copy
+    s = copy.copy(w)
+    s.batch = 1
+    for f in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits"):
+        if getattr(w, f) is not None:
+            setattr(s, f, getattr(w, f)[b:b + 1])
+    s.page_table, s.seq_lens = w.page_table[b:b + 1], w.seq_lens[b:b + 1]
+    return s
+
+
+def cpu_attn_sample(w, seqs):
+    """The CPU checker's verify attention on the given sequences of the workload; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    for b in seqs:
+        s = one_sequence(w, b)
+        oracle.verify_attn(s.q, s.k_tree, s.v_tree, w.k_pool, w.v_pool, s.page_table, s.seq_lens, s.parent, w.scale)
+    return time.perf_counter() - t0
+
+
+def cpu_step_sample(w, seqs):
+    """The CPU checker's whole step (attention, argmax, acceptance, commit) on the given sequences; seconds."""
     import numpy as np
     import oracle
     t0 = time.perf_counter()
     for b in seqs:
-        s = copy.copy(w)
-        s.batch = 1
-        for f in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits"):
-            setattr(s, f, getattr(w, f)[b:b + 1])
-        s.page_table, s.seq_lens = w.page_table[b:b + 1], w.seq_lens[b:b + 1]
+        s = one_sequence(w, b)
         oracle.verify_attn(s.q, s.k_tree, s.v_tree, w.k_pool, w.v_pool, s.page_table, s.seq_lens, s.parent, w.scale)
         tgt = oracle.argmax(s.logits)
         a = oracle.accept(s.parent, s.node_tokens, tgt, w.max_path)
@@ -131,17 +196,25 @@ def cpu_sample_step(w, seqs):
 
 
 def cpu_baseline(w, budget_s=12.0):
-    """The checker as it stands, whole step, sequence after sequence (wrapping around the batch) until
-    about budget_s seconds of CPU work are done."""
+    """The checker as it stands: verify attention, sequence after sequence (wrapping around the batch),
+    until about budget_s seconds of CPU work are done; then a few whole steps for the step's figure."""
     import oracle
     cores = oracle.num_threads()
     done, spent = 0, 0.0
     while spent < budget_s and done < 64 * w.batch:
-        spent += cpu_sample_step(w, [done % w.batch])
+        spent += cpu_attn_sample(w, [done % w.batch])
         done += 1
-    return {"value": done * w.n_nodes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"whole step on {done} sequences drawn in order from the {w.batch} of the workload "
-                      f"({done * w.n_nodes} tree tokens), {spent:.1f} s"}
+    res = {"value": done * w.n_nodes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"verify attention on {done} sequences drawn in order from the {w.batch} of the workload "
+                     f"({done * w.n_nodes} tree tokens), {spent:.1f} s"}
+    if w.logits is not None:
+        n, t = 0, 0.0
+        while t < 3.0 and n < w.batch:
+            t += cpu_step_sample(w, [n])
+            n += 1
+        res["whole_step"] = {"value": n * w.n_nodes / t, "unit": UNIT,
+                             "sample": f"attention + argmax + acceptance + commit on {n} sequences, {t:.1f} s"}
+    return res
 
 
 def run_reference(args):
@@ -151,20 +224,20 @@ def run_reference(args):
     import oracle
     from paper_2508_09072_b200 import workloads as W
     oracle.build()
-    w = W.make(args.workload)
-    t1 = cpu_sample_step(w, [0])                      # also warms the page cache and the library
+    w = W.make(args.workload, with_logits=False)
+    t1 = cpu_attn_sample(w, [0])                      # also warms the page cache and the library
     per_step = 120.0 / (args.steps + args.warmup)     # the whole run should end within a few minutes
     n_seq = int(min(w.batch, max(1, per_step / max(t1, 1e-4))))
     seqs = list(range(n_seq))
     for _ in range(args.warmup):
-        cpu_sample_step(w, seqs)
+        cpu_attn_sample(w, seqs)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        cpu_sample_step(w, seqs)
+        cpu_attn_sample(w, seqs)
     dt = time.perf_counter() - t0
     value = args.steps * n_seq * w.n_nodes / dt
     cores = oracle.num_threads()
-    sample = f"each step = whole path on the first {n_seq} of {w.batch} sequences of {args.workload}"
+    sample = f"each step = verify attention on the first {n_seq} of {w.batch} sequences of {args.workload}"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
@@ -194,6 +267,84 @@ def aggregate_tokens_per_s(batch, tree_nodes, world, steps, ms_max):
     return batch * tree_nodes * world * steps / (ms_max * 1e-3)
 
 
+def blocks_for(t_call_ms: float, steps: int, target_ms: float, cap_calls: int) -> int:
+    """How many blocks of `steps` calls to time so that about target_ms of device time is covered."""
+    per_block = max(t_call_ms * steps, 1e-6)
+    return int(max(1, min(math.ceil(target_ms / per_block), max(1, cap_calls // max(steps, 1)))))
+
+
+# ------------------------------------------------------------------------------------------------
+# verify attention of one workload: kernel alone, isolated call, back-to-back calls
+# ------------------------------------------------------------------------------------------------
+class AttnCase:
+    """One workload on the device with everything a reader_verify_attn call needs."""
+
+    def __init__(self, rd, w, dev, with_logits=False):
+        import torch
+        from paper_2508_09072_b200 import binding
+        self.rd, self.w = rd, w
+        self.d = d = binding.to_device(w, dev, with_logits=with_logits)
+        self.anc, _, enc_status = rd.tree_encode(d.parent)
+        self.out = torch.empty_like(d.q)
+        self.status = torch.empty(w.batch, dtype=torch.int32, device=dev)
+        self.ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
+        assert int(enc_status.max().item()) == 0
+
+    def call(self):
+        d = self.d
+        self.rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, self.w.scale, anc_mask=self.anc, out=self.out,
+                            status=self.status, workspace=self.ws)
+
+
+def attn_row(case: AttnCase, flush, peaks, iters: int, pipelined_ms: float):
+    """Cold-L2 figures of one workload: the attention kernel alone (events inside the call) and the whole
+    call (events around it, its launches overlapping as in production); optionally back-to-back calls."""
+    import torch
+    rd, w = case.rd, case.w
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(5):
+        case.call()
+    tk, tc = [], []
+    for _ in range(iters):
+        flush()
+        c, e = mk(), mk()
+        c.record(); e.record()
+        rd.set_timing_events(c, e)
+        case.call()
+        torch.cuda.synchronize()
+        tk.append(c.elapsed_time(e))
+    rd.set_timing_events(None, None)
+    for _ in range(iters):
+        flush()
+        a, b = mk(), mk()
+        a.record(); case.call(); b.record()
+        torch.cuda.synchronize()
+        tc.append(a.elapsed_time(b))
+    assert int(case.status.max().item()) == 0
+    k, c_ = median(tk) * 1e-3, median(tc) * 1e-3
+    by, fl = w.attn_algorithmic_bytes(), w.attn_algorithmic_flops()
+    t_hbm, t_tc = by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops_sustained"] * 1e12)
+    row = {"workload": w.name, "tokens": w.batch * w.n_nodes, "kernel_us": k * 1e6, "kernel_us_min": min(tk) * 1e3,
+           "call_us": c_ * 1e6, "call_us_min": min(tc) * 1e3, "algorithmic_bytes": by, "algorithmic_flops": fl,
+           "gbs": by / k / 1e9, "hbm_frac": by / k / 1e9 / peaks["hbm_gbs"], "hbm_frac_of_nominal_8tbs": by / k / 8e12,
+           "tflops": fl / k / 1e12, "tensor_frac": fl / k / 1e12 / peaks["bf16_tflops_sustained"],
+           "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
+           "binding_bound": "hbm" if t_hbm >= t_tc else "tensor", "binding_frac": max(t_hbm, t_tc) / k,
+           "binding_frac_call": max(t_hbm, t_tc) / c_, "tokens_per_s": w.batch * w.n_nodes / c_,
+           "l2": "flushed before every call"}
+    if pipelined_ms > 0 and not fits_l2(w):
+        n = max(20, int(pipelined_ms / (c_ * 1e3)))
+        a, b = mk(), mk()
+        a.record()
+        for _ in range(n):
+            case.call()
+        b.record()
+        torch.cuda.synchronize()
+        row["call_us_back_to_back"] = a.elapsed_time(b) / n * 1e3
+        row["tokens_per_s_back_to_back"] = w.batch * w.n_nodes / (a.elapsed_time(b) / n * 1e-3)
+    return row
+
+
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
@@ -216,17 +367,126 @@ def run_ours(args):
     rd = binding.Reader(local)
     if args.kernel:
         rd.set_attn_kernel(args.kernel)
-    d = binding.to_device(w, dev)
+    case = AttnCase(rd, w, dev, with_logits=True)
+    d, out, status, ws = case.d, case.out, case.status, case.ws
     B, T = w.batch, w.n_nodes
+    K, Wm = args.steps, max(args.warmup, 3)
+    small = fits_l2(w)
+    flush_buf = torch.zeros((512 << 20) // 4, dtype=torch.int32, device=dev)
+    flush_sink = torch.zeros((), dtype=torch.int64, device=dev)
+
+    def flush():
+        # a READ pass over four times the L2: the cache ends up holding clean lines of a buffer nobody
+        # uses (a write pass would leave 126 MB of dirty lines to be written back under the next kernel)
+        torch.sum(flush_buf, out=flush_sink)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def mk():
+        return torch.cuda.Event(enable_timing=True)
+
+    # ---- main region: blocks of K reader_verify_attn calls, device-resident inputs
+    for _ in range(Wm):
+        case.call()
+    p0, p1 = mk(), mk()
+    torch.cuda.synchronize()
+    p0.record()
+    for _ in range(10):
+        case.call()
+    p1.record()
+    torch.cuda.synchronize()
+    t_est = p0.elapsed_time(p1) / 10
+    n_blocks = blocks_for(t_est, K, args.min_timed_ms if not small else args.min_timed_ms / 4, 40000 if not small else 8000)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_wall0 = time.time()
+    if not small:
+        marks = [mk() for _ in range(n_blocks + 1)]
+        marks[0].record()
+        for i in range(n_blocks):
+            for _ in range(K):
+                case.call()
+            marks[i + 1].record()
+        barrier()
+        block_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(n_blocks)]
+    else:
+        pairs = [(mk(), mk()) for _ in range(n_blocks * K)]
+        for a, b in pairs:
+            flush()
+            a.record(); case.call(); b.record()
+        barrier()
+        ts = [a.elapsed_time(b) for a, b in pairs]
+        block_ms = [sum(ts[i * K:(i + 1) * K]) for i in range(n_blocks)]
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_block = median(block_ms)
+    assert int(status.max().item()) == 0
+
+    # ---- the attention kernel alone: a second loop with events inside the call around the kernel (events
+    # between two kernels switch the overlap of their launches off, so this loop is a little slower)
+    Kb = max(20, min(300, n_blocks * K))
+    kev = [(mk(), mk()) for _ in range(Kb)]
+    for a, b in kev:                                  # create the handles
+        a.record(); b.record()
+    worst = torch.zeros((), dtype=torch.int32, device=dev)   # a bounded wait that gave up shows in the status words
+    for i in range(Kb):
+        if small:
+            flush()
+        rd.set_timing_events(*kev[i])
+        case.call()
+        worst = torch.maximum(worst, status.max())
+    barrier()
+    rd.set_timing_events(None, None)
+    assert int(worst.item()) == 0, f"status {int(worst.item())} seen during the kernel-timing loop"
+    t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
+
+    # ---- end to end: the step's inputs from pinned host memory, the output back, every call
+    host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent")}
+    host_out = {"out": torch.empty(out.shape, dtype=out.dtype).pin_memory(),
+                "status": torch.empty(B, dtype=torch.int32).pin_memory()}
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_call():
+        for k, t in host_in.items():
+            getattr(d, k).copy_(t, non_blocking=True)
+        rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, out=out, status=status, workspace=ws)
+        host_out["out"].copy_(out, non_blocking=True)
+        host_out["status"].copy_(status, non_blocking=True)
+        torch.cuda.current_stream().synchronize()     # the caller needs the result before the next step
+
+    for _ in range(3):
+        e2e_call()
+    q0, q1 = mk(), mk()
+    q0.record(); e2e_call(); q1.record()
+    torch.cuda.synchronize()
+    ne = blocks_for(q0.elapsed_time(q1), K, args.min_timed_ms / 4, 4000)
+    barrier()
+    e_ms = []
+    for _ in range(ne):
+        f0, f1 = mk(), mk()
+        f0.record()
+        for _ in range(K):
+            e2e_call()
+        f1.record()
+        torch.cuda.synchronize()
+        e_ms.append(f0.elapsed_time(f1))
+    barrier()
+    ms_e2e_block = median(e_ms)
+    assert int(host_out["status"].max().item()) == 0
+
+    # ---- the whole step: attention (masks encoded inside the call), acceptance from logits, commit
     seq_lens0 = d.cache.seq_lens.clone()
-    out = torch.empty_like(d.q)
-    status = torch.empty(B, dtype=torch.int32, device=dev)
     tgt = torch.empty((B, T), dtype=torch.int32, device=dev)
     acc_out = (torch.empty((B, w.max_path), dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
                torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev))
     slots = torch.empty((B, w.max_path), dtype=torch.int32, device=dev)
     cstat = torch.empty(B, dtype=torch.int32, device=dev)
-    ws = rd.workspace(B, T, w.n_q_heads, w.n_kv_heads, w.head_dim)
 
     def step(ev=None):
         d.cache.seq_lens.copy_(seq_lens0)            # harness: rewind the cache length
@@ -239,65 +499,156 @@ def run_ours(args):
                          workspace=ws, outs=acc_out, slots=slots, commit_status=cstat)
         if ev:
             ev[2].record()
-            ev[3].record()
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def mk():
-        return torch.cuda.Event(enable_timing=True)
-
-    # ---- device-resident timing: K steps back to back, nothing but the library's launches in between
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(3):
         step()
-    K = args.steps
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    Ks = max(20, min(300, n_blocks * K))
+    s0, s1 = mk(), mk()
     barrier()
-    t_wall0 = time.time()
-    e0, e1 = mk(), mk()
-    e0.record()
-    for i in range(K):
+    s0.record()
+    for _ in range(Ks):
         step()
-    e1.record()
+    s1.record()
     barrier()
-    t_wall1 = time.time()
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    ms_total = e0.elapsed_time(e1)
-    stall_suspected = False   # set below if the main loop is far slower than the sum of its calls
+    t_step = s0.elapsed_time(s1) / Ks
     assert int(status.max().item()) == 0 and int(cstat.max().item()) == 0 and int(acc_out[3].max().item()) == 0
-
-    # ---- per-call and per-kernel breakdown: a second, shorter loop with events between the calls and,
-    # inside reader_verify_attn, around the attention kernel (events between two kernels switch the
-    # overlap of their launches off, so this loop is a little slower than the one above)
-    Kb = max(3, min(K, 300))
-    evs = [[mk() for _ in range(4)] for _ in range(Kb)]
-    kev = [(mk(), mk()) for _ in range(Kb)]
-    aev = [(mk(), mk()) for _ in range(Kb)]
-    for a, b in kev + aev:                            # create the handles
+    evs = [[mk() for _ in range(3)] for _ in range(Ks)]
+    aev = [(mk(), mk()) for _ in range(Ks)]
+    for a, b in aev:
         a.record(); b.record()
-    worst = torch.zeros((), dtype=torch.int32, device=dev)   # a bounded wait that gave up shows in the status words
-    for i in range(Kb):
-        rd.set_timing_events(*kev[i])
+    for i in range(Ks):
         rd.set_accept_timing_events(*aev[i])
         step(evs[i])
-        worst = torch.maximum(worst, torch.maximum(status.max(), cstat.max()))
     barrier()
-    rd.set_timing_events(None, None)
     rd.set_accept_timing_events(None, None)
-    assert int(worst.item()) == 0, f"status {int(worst.item())} seen during the breakdown loop"
-    t_attn_call = sum(e[0].elapsed_time(e[1]) for e in evs) / Kb
-    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / Kb
-    t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / Kb
-    t_attn_kernel = sum(a.elapsed_time(b) for a, b in kev) / Kb
-    t_argmax_kernel = sum(a.elapsed_time(b) for a, b in aev) / Kb
-    stall_suspected = ms_total / K > 3.0 * (t_attn_call + t_accept + t_commit)
+    t_attn_in_step = sum(e[0].elapsed_time(e[1]) for e in evs) / Ks
+    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / Ks
+    t_argmax_kernel = sum(a.elapsed_time(b) for a, b in aev) / Ks
 
-    # ---- the same step captured once in a CUDA graph and replayed (no host work per step)
-    t_graph = None
+    # reader_kv_commit on its own (the step above runs it inside reader_accept_commit)
+    c_times = []
+    for _ in range(20):
+        d.cache.seq_lens.copy_(seq_lens0)
+        c0, c1 = mk(), mk()
+        c0.record()
+        rd.kv_commit(d.cache, d.k_tree, d.v_tree, acc_out[0], acc_out[1], slots=slots, status=cstat)
+        c1.record()
+        torch.cuda.synchronize()
+        c_times.append(c0.elapsed_time(c1))
+    t_commit = median(c_times)
+    # and the acceptance walk alone, from given target ids
+    a_times = []
+    for _ in range(20):
+        a0, a1 = mk(), mk()
+        a0.record()
+        rd.accept(d.parent, d.node_tokens, w.max_path, target_ids=tgt, outs=acc_out)
+        a1.record()
+        torch.cuda.synchronize()
+        a_times.append(a0.elapsed_time(a1))
+    t_walk = median(a_times)
+
+    extras = {}
+    if not args.quick:
+        extras = run_extras(args, rd, w, d, dev, rank, step, seq_lens0, out, status, ws, tgt, acc_out, slots, cstat, barrier, mk)
+
+    # ---- all five workloads, L2 flushed before every call (rank 0 of a single-GPU run)
+    table = None
+    if world == 1 and not args.no_table:
+        table = []
+        for name in W.WORKLOADS:
+            if name == args.workload:
+                c2 = case
+            else:
+                c2 = AttnCase(rd, W.make(name, with_logits=False), dev)
+            table.append(attn_row(c2, flush, peaks, args.table_iters, 30.0))
+            if c2 is not case:
+                del c2
+                torch.cuda.empty_cache()
+
+    # ---- max over ranks
+    ms_block, ms_e2e_block, t_attn_kernel, t_step, t_accept, t_argmax_kernel, t_commit, t_walk = max_over_ranks(
+        [ms_block, ms_e2e_block, t_attn_kernel, t_step, t_accept, t_argmax_kernel, t_commit, t_walk], dev, world)
+
+    if rank == 0:
+        tokens = B * T * world
+        value = aggregate_tokens_per_s(B, T, world, K, ms_block)
+        e2e = aggregate_tokens_per_s(B, T, world, K, ms_e2e_block)
+        attn_bytes, attn_flops = w.attn_algorithmic_bytes(), w.attn_algorithmic_flops()
+        t_call = ms_block / K
+        t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_tc = attn_flops / (peaks["bf16_tflops_sustained"] * 1e12)
+        bound = "hbm" if t_hbm >= t_tc else "tensor"
+        gbs = attn_bytes / (t_attn_kernel * 1e-3) / 1e9
+        tfs = attn_flops / (t_attn_kernel * 1e-3) / 1e12
+        traffic, traffic_src = ncu_traffic("verify_attn", args.workload)
+        if bound == "hbm":
+            roof = {"kernel": "verify_attn (attn_sm100_kernel)", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": traffic, "traffic_source": traffic_src,
+                    "peak_kind": peak_kind, "frac_of_nominal_8tbs": gbs / 8000.0,
+                    "frac_whole_call": attn_bytes / (t_call * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        else:
+            roof = {"kernel": "verify_attn (attn_sm100_kernel)", "bound": "tensor", "achieved": tfs,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": tfs / peaks["bf16_tflops_sustained"],
+                    "traffic": traffic, "traffic_source": traffic_src, "peak_kind": peak_kind + " (sustained)",
+                    "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"],
+                    "frac_whole_call": attn_flops / (t_call * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]}
+        am_traffic, am_src = ncu_traffic("argmax", args.workload)
+        kernels = {
+            "verify_attn": {"kernel_ms": t_attn_kernel, "call_ms": t_call, "call_ms_in_step": t_attn_in_step,
+                            "algorithmic_bytes": attn_bytes, "gbs": gbs, "algorithmic_flops": attn_flops, "tflops": tfs,
+                            "binding_bound": bound, "binding_frac": max(t_hbm, t_tc) / (t_attn_kernel * 1e-3),
+                            "note": "kernel_ms: attention kernel alone (events inside the call); call_ms: the headline, "
+                                    "one call of back-to-back calls (preparation + attention + combine, launches overlapping)"},
+            "accept": {"argmax_kernel_ms": t_argmax_kernel, "walk_call_ms": t_walk, "accept_commit_call_ms": t_accept,
+                       "algorithmic_bytes": w.logits_bytes(), "gbs": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9,
+                       "hbm_frac": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "traffic": am_traffic, "traffic_source": am_src,
+                       "note": "argmax_kernel_ms / gbs: the target argmax over the logits alone; walk_call_ms: reader_accept "
+                               "from given target ids; accept_commit_call_ms: reader_accept_commit from logits inside the step "
+                               "(argmax, then walk and commit in one launch)"},
+            "kv_commit": {"call_ms": t_commit, "note": "reader_kv_commit alone, one layer"},
+        }
+        kernels.update(extras.get("kernels", {}))
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": t_call, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args.workload),
+            "timed": {"blocks": n_blocks, "steps_per_block": K, "timed_region_ms": sum(block_ms), "block_ms_median": ms_block,
+                      "block_ms_min": min(block_ms), "block_ms_max": max(block_ms),
+                      "note": "a step = one reader_verify_attn call; blocks of `steps` calls repeated until about a second "
+                              "is timed, the median block is reported"},
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "blocks": ne,
+                    "ms_per_step": ms_e2e_block / K},
+            "gpu_launches": LAUNCHES_PER_ATTN_CALL * K * n_blocks, "clocks": clocks, "roofline": roof,
+            "whole_step": {"ms_per_step": t_step, "tokens_per_s": tokens / (t_step * 1e-3), "launches_per_step": LAUNCHES_PER_STEP,
+                           "steps": Ks, "note": "reader_verify_attn (masks encoded inside) + reader_accept_commit from logits, "
+                                                "back to back; reported beside the metric, not folded into it"},
+            "kernels": kernels,
+        }
+        for k in ("cuda_graph_replay", "model_step"):
+            if k in extras:
+                line[k] = extras[k]
+        if table is not None:
+            line["workloads"] = table
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    rd.close()
+
+
+def run_extras(args, rd, w, d, dev, rank, step, seq_lens0, out, status, ws, tgt, acc_out, slots, cstat, barrier, mk):
+    """What surrounds the metric: the step as a CUDA graph, a 32-layer model step, batched commits, the
+    sampling policy's kernel and Algorithm 4 on a padded cache.  None of it enters `value`."""
+    import torch
+    from paper_2508_09072_b200 import binding
+    B, T = w.batch, w.n_nodes
+    res = {"kernels": {}}
+
+    # ---- the whole step captured once in a CUDA graph and replayed (no host work per step)
     try:
         side = torch.cuda.Stream()
         with torch.cuda.stream(side):
@@ -309,7 +660,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         for _ in range(5):
             graph.replay()
-        Kg = max(3, min(K, 500))
+        Kg = 200
         barrier()
         g0, g1 = mk(), mk()
         g0.record()
@@ -318,11 +669,11 @@ def run_ours(args):
         g1.record()
         barrier()
         t_graph = g0.elapsed_time(g1) / Kg
+        res["cuda_graph_replay"] = {"ms_per_step": t_graph, "tokens_per_s": B * T / (t_graph * 1e-3), "what": "the whole step"}
     except Exception as exc:                                  # reported, never hidden
-        t_graph = f"capture failed: {exc}"
+        res["cuda_graph_replay"] = f"capture failed: {exc}"
 
-    # ---- a 32-layer model's commits: layer by layer against one batched launch (pools of one page per
-    # sequence would do for the copy itself; the step's own pool is reused for every layer here)
+    # ---- a 32-layer model's commits: layer by layer against one batched launch
     n_layers = 32
     layer_caches = [d.cache] * n_layers
     lk, lv = [d.k_tree] * n_layers, [d.v_tree] * n_layers
@@ -347,11 +698,12 @@ def run_ours(args):
         c1.record()
         barrier()
         t_layers[label] = c0.elapsed_time(c1) / 20
+    res["kernels"]["kv_commit_32_layers"] = {"call_ms": t_layers, "note": "the accepted rows committed into 32 layers: 32 calls of "
+                                             "reader_kv_commit against one reader_kv_commit_layers"}
 
     # ---- a whole model's verification step: every layer's attention over that layer's own cache (device
     # copies of the pool, one block table for the model), one acceptance, one commit into all layers;
     # issued call by call, then captured once in a CUDA graph and replayed
-    model_step_res = None
     try:
         pool_bytes = 2 * d.cache.k_pool.numel() * d.cache.k_pool.element_size()
         Lm = max(2, min(n_layers, int(40e9 // max(pool_bytes, 1))))
@@ -395,48 +747,41 @@ def run_ours(args):
         t_model_graph = m2.elapsed_time(m3) / 20
         assert int(status.max().item()) == 0 and int(cstat.max().item()) == 0
         kv_bytes = Lm * w.attn_algorithmic_bytes() + w.logits_bytes()
-        model_step_res = {"layers": Lm, "ms_per_step": {"call_by_call": t_model_eager, "cuda_graph": t_model_graph},
-                          "tokens_per_s": B * T / (t_model_graph * 1e-3), "algorithmic_bytes": kv_bytes,
-                          "gbs": kv_bytes / (t_model_graph * 1e-3) / 1e9,
-                          "note": "checks and work partition once, every layer's verify attention on its own cache, one acceptance, one commit into all layers; "
-                                  "not the metric's step (one layer), reported beside it"}
+        best = min(t_model_eager, t_model_graph)
+        res["model_step"] = {"layers": Lm, "ms_per_step": {"call_by_call": t_model_eager, "cuda_graph": t_model_graph},
+                             "ms_per_layer": (best - 0.0) / Lm, "tokens_per_s": B * T / (best * 1e-3), "algorithmic_bytes": kv_bytes,
+                             "gbs": kv_bytes / (best * 1e-3) / 1e9,
+                             "note": "checks and work partition once, every layer's verify attention on its own cache, one "
+                                     "acceptance, one commit into all layers; reported beside the metric"}
         del m_caches, mgraph
+        torch.cuda.empty_cache()
     except Exception as exc:                                  # reported, never hidden
-        model_step_res = f"failed: {exc}"
+        res["model_step"] = f"failed: {exc}"
 
     # ---- the sampling policy's target kernel (an alternative to the argmax; not part of the step)
     uni = torch.rand((B, T), dtype=torch.float32, device=dev)
     tgt_s = torch.empty((B, T), dtype=torch.int32, device=dev)
-    for _ in range(3):
-        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s)
-    s0, s1 = mk(), mk()
-    s0.record()
-    for _ in range(20):
-        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s)
-    s1.record()
-    barrier()
-    t_sample = s0.elapsed_time(s1) / 20
-    s2, s3 = mk(), mk()
-    rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, top_k=50)
-    s2.record()
-    for _ in range(10):
-        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, top_k=50)
-    s3.record()
-    barrier()
-    t_sample_topk = s2.elapsed_time(s3) / 10
-    t_sample_variants = {}
-    for label, kw in (("top_p_0.9", dict(top_p=0.9)), ("top_k_50_top_p_0.9", dict(top_k=50, top_p=0.9))):
-        rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, **kw)
-        v0, v1 = mk(), mk()
-        v0.record()
-        for _ in range(5):
+
+    def time_sample(n, **kw):
+        for _ in range(2):
             rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, **kw)
-        v1.record()
+        a, b = mk(), mk()
+        a.record()
+        for _ in range(n):
+            rd.sample_targets(d.parent, d.logits, uni, 0.8, target_ids=tgt_s, **kw)
+        b.record()
         barrier()
-        t_sample_variants[label] = v0.elapsed_time(v1) / 5
+        return a.elapsed_time(b) / n
+
+    t_sample = time_sample(20)
+    res["kernels"]["sample_targets"] = {
+        "call_ms": t_sample, "algorithmic_bytes": w.logits_bytes(), "gbs": w.logits_bytes() / (t_sample * 1e-3) / 1e9,
+        "variants_call_ms": {"top_k_50": time_sample(10, top_k=50), "top_p_0.9": time_sample(5, top_p=0.9),
+                             "top_k_50_top_p_0.9": time_sample(5, top_k=50, top_p=0.9)},
+        "note": "sampling policy (Appendix C, temperature 0.8); replaces the argmax when used; flat synthetic logits, so "
+                "the nucleus for 0.9 holds tens of thousands of tokens"}
 
     # ---- the paper's own cache maintenance (Algorithm 4) on a padded batch cache of the same size class
-    # (not part of the step: the paged cache needs no such pass)
     capR, gen = 4096, torch.Generator(device=dev)
     gen.manual_seed(1234 + rank)
     kR = torch.randn((B, w.n_kv_heads, capR, w.head_dim), device=dev, generator=gen).to(torch.bfloat16)
@@ -452,107 +797,13 @@ def run_ours(args):
         r0.record(); rd.kv_rearrange(kR, vR, maskR, lenR); r1.record()
         torch.cuda.synchronize()
         r_times.append(r0.elapsed_time(r1))
-    t_rearr = sorted(r_times)[len(r_times) // 2]
+    t_rearr = median(r_times)
     rearr_bytes = 2 * 2 * (B * w.n_kv_heads * (capR - capR // 2) * w.head_dim * 2)   # K and V, read + write of the moving half
+    res["kernels"]["kv_rearrange"] = {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,
+                                      "note": "Algorithm 4 on a padded batch cache [B][Hkv][4096][D], 85 % valid behind a compact "
+                                              "first half"}
     del kR, vR
-
-    # ---- end to end: host buffers in, results out, every step
-    host_in = {k: getattr(d, k).cpu().pin_memory() for k in ("q", "k_tree", "v_tree", "parent", "node_tokens", "logits")}
-    host_out = {"out": torch.empty(out.shape, dtype=out.dtype).pin_memory(),
-                "path": torch.empty(acc_out[0].shape, dtype=torch.int32).pin_memory(),
-                "n_acc": torch.empty(B, dtype=torch.int32).pin_memory(),
-                "bonus": torch.empty(B, dtype=torch.int32).pin_memory(),
-                "slots": torch.empty(slots.shape, dtype=torch.int32).pin_memory()}
-    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
-    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
-
-    def e2e_step():
-        for k, t in host_in.items():
-            getattr(d, k).copy_(t, non_blocking=True)
-        step()
-        host_out["out"].copy_(out, non_blocking=True)
-        host_out["path"].copy_(acc_out[0], non_blocking=True)
-        host_out["n_acc"].copy_(acc_out[1], non_blocking=True)
-        host_out["bonus"].copy_(acc_out[2], non_blocking=True)
-        host_out["slots"].copy_(slots, non_blocking=True)
-        torch.cuda.current_stream().synchronize()     # the caller needs the result before the next step
-
-    Ke = max(3, min(K, args.e2e_steps))
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    f0, f1 = mk(), mk()
-    f0.record()
-    for _ in range(Ke):
-        e2e_step()
-    f1.record()
-    barrier()
-    ms_e2e = f0.elapsed_time(f1)
-
-    # ---- max over ranks
-    ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel, t_argmax_kernel = max_over_ranks(
-        [ms_total, ms_e2e, t_attn_call, t_accept, t_commit, t_attn_kernel, t_argmax_kernel], dev, world)
-
-    if rank == 0:
-        tokens = B * T * world
-        value = aggregate_tokens_per_s(B, T, world, K, ms_total)
-        e2e = aggregate_tokens_per_s(B, T, world, Ke, ms_e2e)
-        attn_bytes = w.attn_algorithmic_bytes()
-        attn_flops = w.attn_algorithmic_flops()
-        kernels = {
-            "verify_attn": {"ms": t_attn_kernel, "call_ms": t_attn_call, "algorithmic_bytes": attn_bytes,
-                            "gbs": attn_bytes / (t_attn_kernel * 1e-3) / 1e9,
-                            "algorithmic_flops": attn_flops, "tflops": attn_flops / (t_attn_kernel * 1e-3) / 1e12,
-                            "tokens_per_s_call": tokens / (t_attn_call * 1e-3)},
-            "accept": {"ms": t_argmax_kernel, "call_ms": t_accept, "algorithmic_bytes": w.logits_bytes(),
-                       "gbs": w.logits_bytes() / (t_argmax_kernel * 1e-3) / 1e9,
-                       "note": "ms / gbs: the argmax kernel alone; call_ms is reader_accept_commit: it adds the acceptance walk "
-                               "and the KV commit, which share one launch"},
-            "kv_commit_32_layers": {"call_ms": t_layers, "note": "the accepted rows committed into 32 layers: 32 calls of "
-                                    "reader_kv_commit against one reader_kv_commit_layers; not in the step"},
-            "kv_rearrange": {"call_ms": t_rearr, "moved_bytes": rearr_bytes, "gbs": rearr_bytes / (t_rearr * 1e-3) / 1e9,
-                             "note": "Algorithm 4 on a padded batch cache [B][Hkv][4096][D], 85 % valid behind a compact "
-                                     "first half; not in the step"},
-            "sample_targets": {"call_ms": t_sample, "algorithmic_bytes": w.logits_bytes(),
-                               "gbs": w.logits_bytes() / (t_sample * 1e-3) / 1e9,
-                               "note": "sampling policy (Appendix C); replaces the argmax when used; not in the step"},
-            "sample_targets_top_p": {"call_ms": t_sample_variants,
-                                     "note": "flat synthetic logits: the nucleus for 0.9 does not fit the candidate list, "
-                                             "so top-p alone selects on the whole row (the slow path)"},
-            "sample_targets_top_k_50": {"call_ms": t_sample_topk, "note": "same with top-k filtering (one more pass over the logits for k <= 256)"},
-        }
-        t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
-        t_tc = attn_flops / (peaks["bf16_tflops_sustained"] * 1e12)
-        kernels["verify_attn"]["binding_bound"] = "hbm" if t_hbm >= t_tc else "tensor"
-        kernels["verify_attn"]["binding_frac"] = max(t_hbm, t_tc) / (t_attn_kernel * 1e-3)
-        def hbm_roof(kernel, gbs):
-            return {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get((kernel, args.workload)),
-                    "peak_kind": peak_kind}
-        roof_attn = hbm_roof("verify_attn", kernels["verify_attn"]["gbs"])
-        if kernels["verify_attn"]["binding_bound"] == "tensor":
-            tf = kernels["verify_attn"]["tflops"]
-            roof_attn = {"kernel": "verify_attn", "bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"],
-                         "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"], "traffic": None,
-                         "peak_kind": peak_kind + " (sustained)"}
-        # the step's dominant kernel; the attention kernel's own roofline is always reported beside it
-        roof = roof_attn if t_attn_kernel >= t_argmax_kernel else hbm_roof("accept (target argmax)", kernels["accept"]["gbs"])
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args.workload),
-            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke},
-            "cuda_graph_replay": ({"ms_per_step": t_graph, "value": B * T * world / (t_graph * 1e-3)} if isinstance(t_graph, float) else t_graph), "model_step": model_step_res, "stall_suspected": bool(stall_suspected), "gpu_launches": LAUNCHES_PER_STEP * K, "clocks": clocks, "roofline": roof, "roofline_verify_attn": roof_attn,
-            "kernels": kernels,
-        }
-        if world == 1 and not args.no_cpu_baseline:
-            import oracle
-            oracle.build()
-            line["cpu_baseline"] = cpu_baseline(w)
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
-    rd.close()
+    return res
 
 
 # ------------------------------------------------------------------------------------------------

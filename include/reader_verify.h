@@ -106,14 +106,18 @@ typedef struct {
 } reader_tree;
 
 /* Creates a context for CUDA device `device` (host call; may initialise the CUDA context).
- * *out is host memory owned by the library until reader_destroy. */
+ * *out is host memory owned by the library until reader_destroy.  READER_ERR_UNSUPPORTED when the
+ * device is not of compute capability 10.x or the tensor-core attention kernel cannot be set up on it
+ * (no tensor-map encoder in the driver, too little shared memory): the library never serves calls
+ * from a slower path on its own. */
 reader_status reader_create(reader_ctx **out, int device);
 void reader_destroy(reader_ctx *ctx);
 const char *reader_status_string(reader_status s);
 
-/* Chooses the attention kernel: 0 = automatic (tensor-core kernel where the shape allows, else
- * the CUDA-core kernel), 1 = always the CUDA-core kernel, 2 = tensor-core kernel or
- * READER_ERR_UNSUPPORTED.  Both compute Sec. 3.2's attention; this is a testing aid. Host call. */
+/* Chooses the attention kernel: 0 = automatic (the tensor-core kernel; the CUDA-core kernel only for
+ * the shapes the former is not built for: a GQA group that does not divide 128, a non-positive
+ * scale), 1 = always the CUDA-core kernel, 2 = tensor-core kernel or READER_ERR_UNSUPPORTED.
+ * Both compute Sec. 3.2's attention; this is a testing aid. Host call. */
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
 
 /* Profiling aid (host call): when both are non-NULL cudaEvent_t handles, the next calls of
@@ -369,6 +373,7 @@ reader_status reader_padded_rearrange(reader_ctx *ctx, reader_padded_cache *cach
  *   - All calls share the array and leave their pairs in it.  Nothing in it needs clearing, every
  *     slot read is written earlier in the same call; but calls that can overlap on the GPU (two
  *     streams, two host threads) race on it -- issue them on one stream or order them.
+ *   - The events of reader_set_accept_timing_events are not recorded by this call.
  */
 reader_status reader_accept_noalloc(reader_ctx *ctx, const reader_tree *tree, const int32_t *node_tokens,
                                     const float *logits, int32_t vocab, int32_t *target_ids,

@@ -27,7 +27,7 @@
 namespace {
 
 constexpr int kMaxRows = READER_NOALLOC_MAX_ROWS;
-constexpr int kSplitsCap = 64;
+constexpr int kSplitsCap = reader::kMaxArgmaxSplits;   // the array holds that many pairs per row
 constexpr size_t kScratchBytes = (size_t)kMaxRows * kSplitsCap * (sizeof(float) + sizeof(int32_t));
 
 // Device-side storage.  In host code this name is only a handle for the runtime's symbol lookup,
@@ -74,23 +74,16 @@ extern "C" reader_status reader_accept_noalloc(reader_ctx *ctx, const reader_tre
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return READER_ERR_CUDA;
     if (dev != ctx->device) return READER_ERR_INVALID_ARG;
-    if (B == 0) return READER_OK;
     unsigned char *scratch = nullptr;
     if (reader_status st = scratch_for_device(dev, &scratch)) return st;
 
-    // enough blocks to fill the GPU, at least 2048 columns each, never more than the array holds
-    int64_t splits = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;
-    if (splits < 3) splits = 3;   // as in reader_accept: never one block per row
-    const int64_t by_width = vocab / 2048 > 0 ? vocab / 2048 : 1;
-    if (splits > by_width) splits = by_width;
-    if (splits > kSplitsCap) splits = kSplitsCap;
-    if (splits < 1) splits = 1;
+    const int splits = argmax_splits(ctx->n_sm, rows, vocab);   // the same cut as reader_accept; <= kSplitsCap
     float *part_val = reinterpret_cast<float *>(scratch);
     int32_t *part_idx = reinterpret_cast<int32_t *>(scratch + (size_t)kMaxRows * kSplitsCap * sizeof(float));
 
     cudaStream_t st = (cudaStream_t)stream;
-    launch_argmax(logits, rows, vocab, (int)splits, part_val, part_idx, st);
-    launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, part_val, part_idx, (int)splits, path_out,
+    launch_argmax(logits, rows, vocab, splits, part_val, part_idx, st);
+    launch_accept(tree->parent, node_tokens, target_ids, B, T, max_path, part_val, part_idx, splits, path_out,
                   n_acc_out, bonus_out, status_out, st);
     return cudaGetLastError() == cudaSuccess ? READER_OK : READER_ERR_CUDA;
 }

@@ -11,7 +11,7 @@ namespace {
 
 using namespace reader;
 
-constexpr int kMaxSplits = 64;
+constexpr int kMaxSplits = kMaxArgmaxSplits;
 constexpr size_t kAlign = 256;
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -50,17 +50,6 @@ inline reader_status check_device(const reader_ctx *ctx) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return READER_ERR_CUDA;
     return dev == ctx->device ? READER_OK : READER_ERR_INVALID_ARG;
-}
-
-// Column ranges a logits row is cut into so that small batches still fill the GPU (>= 2048 columns each).
-inline int argmax_splits(const reader_ctx *ctx, int64_t rows, int64_t vocab) {
-    int64_t want = (4 * (int64_t)ctx->n_sm + rows - 1) / rows;   // enough blocks to fill the GPU when rows are few
-    if (want < 3) want = 3;   // and never one block per row: on C3 three blocks per row took 6 us off the 92 us scan
-    const int64_t cap = vocab / 2048 > 0 ? vocab / 2048 : 1;
-    if (want < 1) want = 1;
-    if (want > cap) want = cap;
-    if (want > kMaxSplits) want = kMaxSplits;
-    return (int)want;
 }
 
 inline reader_status launch_status() { return cudaGetLastError() == cudaSuccess ? READER_OK : READER_ERR_CUDA; }
@@ -426,7 +415,6 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
     const int B = tree->batch, T = tree->n_nodes;
     if (B < 0 || T < 1 || T > kMaxNodes || max_path < 1) return READER_ERR_INVALID_ARG;
     if (reader_status st = check_device(ctx)) return st;
-    if (B == 0) return READER_OK;
     cudaStream_t st = (cudaStream_t)stream;
     int splits = 0;
     float *pv = nullptr;
@@ -438,7 +426,7 @@ reader_status reader_accept(reader_ctx *ctx, const reader_tree *tree, const int3
         const WsLayout w = ws_layout(ctx, B, T, 64);
         if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
         const int64_t rows = (int64_t)B * T;
-        splits = argmax_splits(ctx, rows, vocab);
+        splits = argmax_splits(ctx->n_sm, rows, vocab);
         unsigned char *ws = static_cast<unsigned char *>(workspace);
         pv = reinterpret_cast<float *>(ws + w.amax_val);
         pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);
@@ -478,7 +466,7 @@ reader_status reader_accept_commit(reader_ctx *ctx, const reader_tree *tree, con
             return READER_ERR_INVALID_ARG;
         const WsLayout w = ws_layout(ctx, B, T, 64);
         if (workspace_bytes < w.total) return READER_ERR_WORKSPACE;
-        splits = argmax_splits(ctx, (int64_t)B * T, vocab);
+        splits = argmax_splits(ctx->n_sm, (int64_t)B * T, vocab);
         unsigned char *ws = static_cast<unsigned char *>(workspace);
         pv = reinterpret_cast<float *>(ws + w.amax_val);
         pi = reinterpret_cast<int32_t *>(ws + w.amax_idx);

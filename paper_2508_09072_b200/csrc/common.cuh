@@ -270,6 +270,20 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Column ranges a logits row is cut into by the argmax scan (reader_accept, reader_accept_commit,
+// reader_accept_noalloc): enough blocks to fill the GPU when rows are few, at least three per row (one
+// 513 KB block per row left the scan short of bytes in flight), at least 2048 columns each, at most
+// kMaxArgmaxSplits (what the partial arrays are sized for).
+constexpr int kMaxArgmaxSplits = 64;
+inline int argmax_splits(int n_sm, int64_t rows, int64_t vocab) {
+    int64_t want = (4 * (int64_t)n_sm + rows - 1) / rows;
+    if (want < 3) want = 3;
+    const int64_t cap = vocab / 2048 > 0 ? vocab / 2048 : 1;
+    if (want > cap) want = cap;
+    if (want > kMaxArgmaxSplits) want = kMaxArgmaxSplits;
+    return (int)want;
+}
+
 // Host-side launchers (one per .cu file)
 void launch_tree_encode(const int32_t *parent, int B, int T, uint64_t *anc, int32_t *level,
                         int32_t *status, cudaStream_t st);

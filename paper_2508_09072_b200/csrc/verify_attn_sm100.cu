@@ -707,6 +707,9 @@ struct Sm100Maps {
     alignas(64) CUtensorMap ktmap, vtmap, qmap;
 };
 
+// The tensor-core kernel is the library's attention path: a device on which it cannot run (no
+// cuTensorMapEncodeTiled in the driver, too little opt-in shared memory) is refused here, so that no call
+// is ever served silently by the CUDA-core kernel.
 reader_status sm100_host_init(Sm100Host *h, int device) {
     h->encode_tiled = nullptr;
     h->smem_optin = 0;
@@ -716,17 +719,19 @@ reader_status sm100_host_init(Sm100Host *h, int device) {
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess) {
+        q != cudaDriverEntryPointSuccess || !fn) {
         cudaGetLastError();
-        return READER_OK;   // the CUDA-core kernel still serves every shape
+        return READER_ERR_UNSUPPORTED;
     }
     if (cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
         cudaGetLastError();
-        return READER_OK;
+        return READER_ERR_CUDA;
     }
+    if (h->smem_optin < Cfg<128>::kSmemBytes) return READER_ERR_UNSUPPORTED;
     h->maps = new (std::nothrow) Sm100Maps();
+    if (!h->maps) return READER_ERR_CUDA;
     h->encode_tiled = fn;
-    h->ready = h->maps != nullptr && h->smem_optin >= Cfg<128>::kSmemBytes;
+    h->ready = true;
     return READER_OK;
 }
 

@@ -1,4 +1,4 @@
-"""reader_accept_noalloc against reader_accept.
+"""reader_accept_noalloc against reader_accept and against the CPU oracle.
 
 Some hosts cannot give the library a workspace: their device memory is owned by another
 allocator, or they may not make allocating calls where they invoke the acceptance step.  The
@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2508_09072_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -42,6 +43,12 @@ def test_noalloc_accept_equals_accept_on_two_calls_in_a_row():
             for k in ("target_ids", "path", "n_acc", "bonus", "status"):
                 np.testing.assert_array_equal(got[k], ref[k], err_msg=f"{w.name}:{k}")   # integers: exact
             assert (ref["n_acc"] >= 1).all()
+            # and against the definition itself: first index of the row maximum, longest consistent root path
+            tgt = oracle.argmax(w.logits)
+            np.testing.assert_array_equal(got["target_ids"], tgt, err_msg=f"{w.name}: target ids vs oracle")
+            want = oracle.accept(w.parent, w.node_tokens, tgt, w.max_path)
+            for k in ("path", "n_acc", "bonus", "status"):
+                np.testing.assert_array_equal(got[k], want[k], err_msg=f"{w.name}:{k} vs oracle")
     finally:
         rd.close()
 
