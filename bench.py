@@ -378,7 +378,7 @@ def run_ours(args):
     def flush():
         # a READ pass over four times the L2: the cache ends up holding clean lines of a buffer nobody
         # uses (a write pass would leave 126 MB of dirty lines to be written back under the next kernel)
-        torch.sum(flush_buf, out=flush_sink)
+        torch.sum(flush_buf, dim=(0,), out=flush_sink)
 
     def barrier():
         if world > 1:
@@ -816,7 +816,7 @@ def run_sweep(args):
     from paper_2508_09072_b200 import binding, workloads as W
     torch.cuda.set_device(0)
     rd = binding.Reader(0)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = make_flush()
     peaks, _ = load_peaks()
     rows = []
     for B in (1, 8, 32):
@@ -837,7 +837,7 @@ def run_sweep(args):
                 call()
             ts = []
             for _ in range(args.sweep_iters):
-                flush.zero_()                                  # cold L2: the small cases fit in it
+                flush()                                        # cold L2: the small cases fit in it
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(); call(); b.record()
                 torch.cuda.synchronize()
@@ -856,53 +856,30 @@ def run_sweep(args):
 # ------------------------------------------------------------------------------------------------
 # verify attention alone on all five workloads (cold L2): the numbers behind the roofline table
 # ------------------------------------------------------------------------------------------------
+def make_flush(dev="cuda"):
+    """A read pass over 512 MB (four times the L2): see run_ours."""
+    import torch
+    buf = torch.zeros((512 << 20) // 4, dtype=torch.int32, device=dev)
+    sink = torch.zeros((), dtype=torch.int64, device=dev)
+    return lambda: torch.sum(buf, dim=(0,), out=sink)
+
+
 def run_attn_table(args):
     import torch
     from paper_2508_09072_b200 import binding, workloads as W
     torch.cuda.set_device(0)
     rd = binding.Reader(0)
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    if args.kernel:
+        rd.set_attn_kernel(args.kernel)
+    flush = make_flush()
     peaks, peak_kind = load_peaks()
-    mk = lambda: torch.cuda.Event(enable_timing=True)
     rows = []
-    for name in ("c1", "c2", "c3", "c4", "c5"):
-        w = W.make(name, with_logits=False)
-        d = binding.to_device(w, with_logits=False)
-        anc, _, _ = rd.tree_encode(d.parent)
-        out = torch.empty_like(d.q)
-        st = torch.empty(w.batch, dtype=torch.int32, device="cuda")
-        ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
-        call = lambda: rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out,
-                                      status=st, workspace=ws)
-        for _ in range(5):
-            call()
-        tk, tc = [], []
-        for _ in range(args.sweep_iters):                     # kernel alone (events inside the call)
-            flush.zero_()
-            c, e = mk(), mk()
-            c.record(); e.record()
-            rd.set_timing_events(c, e)
-            call()
-            torch.cuda.synchronize()
-            tk.append(c.elapsed_time(e))
-        rd.set_timing_events(None, None)
-        for _ in range(args.sweep_iters):                     # whole call, launches overlapping as in production
-            flush.zero_()
-            a, b = mk(), mk()
-            a.record(); call(); b.record()
-            torch.cuda.synchronize()
-            tc.append(a.elapsed_time(b))
-        assert int(st.max().item()) == 0
-        k, c_ = sorted(tk)[len(tk) // 2] * 1e-3, sorted(tc)[len(tc) // 2] * 1e-3
-        by, fl = w.attn_algorithmic_bytes(), w.attn_algorithmic_flops()
-        t_hbm, t_tc = by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops_sustained"] * 1e12)
-        rows.append({"workload": name, "kernel_us": k * 1e6, "call_us": c_ * 1e6, "algorithmic_bytes": by,
-                     "algorithmic_flops": fl, "gbs": by / k / 1e9, "hbm_frac": by / k / 1e9 / peaks["hbm_gbs"],
-                     "tflops": fl / k / 1e12, "tensor_frac": fl / k / 1e12 / peaks["bf16_tflops_sustained"],
-                     "binding_bound": "hbm" if t_hbm >= t_tc else "tensor", "binding_frac": max(t_hbm, t_tc) / k,
-                     "tokens_per_s_call": w.batch * w.n_nodes / c_})
-        del d, out
-    print(json.dumps({"table": "verify attention per workload, L2 flushed before every call, median", "peaks": peaks,
+    for name in W.WORKLOADS:
+        case = AttnCase(rd, W.make(name, with_logits=False), "cuda:0")
+        rows.append(attn_row(case, flush, peaks, args.table_iters, 30.0))
+        del case
+        torch.cuda.empty_cache()
+    print(json.dumps({"table": "verify attention per workload, L2 flushed (read pass) before every call, median", "peaks": peaks,
                       "peak_kind": peak_kind, "rows": rows}))
     rd.close()
 
@@ -979,14 +956,14 @@ def run_cache_sim(args):
         return a.elapsed_time(b), int(peak.item()), int(cache.extent.item())
 
     # the same attention call on the two layouts while they still hold the same compact content
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    flush = make_flush()
 
     def call_us(call):
         for _ in range(3):
             call()
         ts = []
         for _ in range(args.sweep_iters):
-            flush.zero_()
+            flush()
             a, b = mk(), mk()
             a.record(); call(); b.record()
             torch.cuda.synchronize()
@@ -1034,12 +1011,15 @@ def run_cache_sim(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--kernel", type=int, default=0, help="attention kernel: 0 auto, 1 CUDA-core, 2 tensor-core")
-    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--min-timed-ms", type=float, default=1000.0, help="blocks of --steps calls are repeated until about this much is timed")
+    ap.add_argument("--table-iters", type=int, default=15, help="calls per measurement in the five-workload table")
+    ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
+    ap.add_argument("--quick", action="store_true", help="skip what surrounds the metric (graph, model step, sampling, rearrangement)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-tree", action="store_true", help="measure the attention call for several tree sizes instead")
     ap.add_argument("--sweep-iters", type=int, default=15)
