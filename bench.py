@@ -565,6 +565,10 @@ def run_ours(args):
                 del c2
                 torch.cuda.empty_cache()
 
+    long_prefix = None
+    if world == 1 and not args.no_table:
+        long_prefix = long_prefix_rows(rd, dev, peaks, args.table_iters)
+
     # ---- max over ranks
     ms_block, ms_e2e_block, t_attn_kernel, t_step, t_accept, t_argmax_kernel, t_commit, t_walk = max_over_ranks(
         [ms_block, ms_e2e_block, t_attn_kernel, t_step, t_accept, t_argmax_kernel, t_commit, t_walk], dev, world)
@@ -630,6 +634,8 @@ def run_ours(args):
                 line[k] = extras[k]
         if table is not None:
             line["workloads"] = table
+        if long_prefix is not None:
+            line["shared_prefix_larger_than_l2"] = long_prefix
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
@@ -885,6 +891,54 @@ def run_attn_table(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# a shared prefix that does not fit the L2: the equal-range partition against the aligned one
+# ------------------------------------------------------------------------------------------------
+def long_prefix_rows(rd, dev, peaks, iters, partitions=(1, 2)):
+    """16 sequences over one 32 768-token prefix (134 MB of K and V) plus private suffixes: attention kernel
+    time under both work partitions.  How often the prefix comes from HBM is in the ncu summary under
+    profiles/ (counters need the profiler); here only times."""
+    import torch
+    from paper_2508_09072_b200 import workloads as W
+    case = AttnCase(rd, W.make_long_shared_prefix(), dev)
+    w = case.w
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    rows = []
+    for part in partitions:
+        rd.set_partition(part)
+        for _ in range(3):
+            case.call()
+        ts = []
+        for _ in range(iters):
+            c, e = mk(), mk()
+            c.record(); e.record()
+            rd.set_timing_events(c, e)
+            case.call()
+            torch.cuda.synchronize()
+            ts.append(c.elapsed_time(e))
+        rd.set_timing_events(None, None)
+        assert int(case.status.max().item()) == 0
+        k = median(ts) * 1e-3
+        by, fl = w.attn_algorithmic_bytes(), w.attn_algorithmic_flops()
+        rows.append({"partition": {1: "equal ranges", 2: "aligned (the automatic choice at this size)"}[part], "kernel_us": k * 1e6,
+                     "algorithmic_bytes": by, "gbs": by / k / 1e9, "algorithmic_flops": fl, "tflops": fl / k / 1e12,
+                     "tensor_frac": fl / k / 1e12 / peaks["bf16_tflops_sustained"]})
+    rd.set_partition(0)
+    return {"workload": "16 sequences sharing a 32768-token prefix (134 MB of K+V) + private suffixes of 256..1024, 32-node trees",
+            "l2": "no flush: every call streams more K/V than the 126 MB L2 holds", "rows": rows}
+
+
+def run_long_prefix(args):
+    import torch
+    from paper_2508_09072_b200 import binding
+    torch.cuda.set_device(0)
+    rd = binding.Reader(0)
+    peaks, _ = load_peaks()
+    parts = (1, 2) if args.partition == 0 else (args.partition,)
+    print(json.dumps(long_prefix_rows(rd, "cuda:0", peaks, args.table_iters, parts)))
+    rd.close()
+
+
+# ------------------------------------------------------------------------------------------------
 # the paper's padded batch cache against the paged cache over a run of decoding steps (Sec. 4.3)
 # ------------------------------------------------------------------------------------------------
 def run_cache_sim(args):
@@ -1024,6 +1078,8 @@ def main():
     ap.add_argument("--sweep-tree", action="store_true", help="measure the attention call for several tree sizes instead")
     ap.add_argument("--sweep-iters", type=int, default=15)
     ap.add_argument("--attn-table", action="store_true", help="verify attention alone on C1..C5 instead")
+    ap.add_argument("--long-prefix", action="store_true", help="a shared prefix larger than L2 under both work partitions instead")
+    ap.add_argument("--partition", type=int, default=0, help="with --long-prefix: 1 equal ranges only, 2 aligned only")
     ap.add_argument("--cache-sim", action="store_true", help="paged cache against the paper's padded batch cache over many steps instead")
     ap.add_argument("--sim-steps", type=int, default=200)
     args = ap.parse_args()
@@ -1031,6 +1087,8 @@ def main():
         run_attn_table(args)
     elif args.cache_sim:
         run_cache_sim(args)
+    elif args.long_prefix:
+        run_long_prefix(args)
     elif args.sweep_tree:
         run_sweep(args)
     elif args.impl == "reference":

@@ -120,6 +120,14 @@ const char *reader_status_string(reader_status s);
  * Both compute Sec. 3.2's attention; this is a testing aid. Host call. */
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
 
+/* Chooses how reader_verify_attn divides its work among thread blocks: 0 = automatic, 1 = always equal
+ * ranges of the flattened tile list (best balance), 2 = the aligned partition whenever a prefix is
+ * shared (every KV stream cut at the same relative positions, so that the sequences sharing a prefix
+ * walk it in step and a prefix larger than the L2 cache is fetched from HBM once; automatic above 48 MB
+ * of shared K and V).  Results do not depend on the choice beyond rounding; this is a testing and
+ * measuring aid.  Host call. */
+reader_status reader_set_partition(reader_ctx *ctx, int32_t which);
+
 /* Profiling aid (host call): when both are non-NULL cudaEvent_t handles, the next calls of
  * reader_verify_attn (and of its prepared and padded forms) record `start` on the stream right before the main attention kernel and
  * `stop` right after it (the preparation and combine kernels lie outside).  NULL, NULL turns it off. */

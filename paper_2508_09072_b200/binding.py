@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libreader_verify.so")
  ERR_TOO_LARGE) = range(10)
 NOALLOC_MAX_ROWS = 4096
 
-EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel",
+EXPORTS = ("reader_create", "reader_destroy", "reader_status_string", "reader_set_attn_kernel", "reader_set_partition",
            "reader_set_timing_events", "reader_set_accept_timing_events",
            "reader_workspace_bytes", "reader_tree_encode", "reader_verify_attn", "reader_accept",
            "reader_kv_commit", "reader_accept_noalloc", "reader_sample_targets", "reader_kv_rearrange", "reader_kv_commit_layers",
@@ -70,6 +70,8 @@ def load_library() -> ctypes.CDLL:
     lib.reader_status_string.restype = ctypes.c_char_p
     lib.reader_set_attn_kernel.argtypes = [c_void_p, c_int32]
     lib.reader_set_attn_kernel.restype = c_int32
+    lib.reader_set_partition.argtypes = [c_void_p, c_int32]
+    lib.reader_set_partition.restype = c_int32
     lib.reader_set_timing_events.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.reader_set_timing_events.restype = c_int32
     lib.reader_set_accept_timing_events.argtypes = [c_void_p, c_void_p, c_void_p]
@@ -211,6 +213,12 @@ class Reader:
         st = self.lib.reader_set_attn_kernel(self._h, int(which))
         if st != OK:
             raise ReaderError(st, "reader_set_attn_kernel")
+
+    def set_partition(self, which: int) -> None:
+        """0 automatic, 1 equal ranges, 2 aligned partition whenever a prefix is shared."""
+        st = self.lib.reader_set_partition(self._h, int(which))
+        if st != OK:
+            raise ReaderError(st, "reader_set_partition")
 
     def set_timing_events(self, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
         """Events (created with enable_timing=True and already recorded once, so that their handles

@@ -12,6 +12,7 @@ namespace {
 using namespace reader;
 
 constexpr int kMaxSplits = kMaxArgmaxSplits;
+constexpr int64_t kAlignedPrefixBytes = 48ll << 20;   // shared prefix K+V above which the lanes walk it in step (L2: 126 MB)
 constexpr size_t kAlign = 256;
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -73,6 +74,7 @@ reader_status reader_create(reader_ctx **out, int device) {
     ctx->device = device;
     ctx->n_sm = n_sm;
     ctx->attn_kernel = 0;
+    ctx->partition = 0;
     ctx->ev_start = ctx->ev_stop = nullptr;
     ctx->ev_acc_start = ctx->ev_acc_stop = nullptr;
     ctx->prepared = PreparedRecord{};
@@ -110,6 +112,12 @@ const char *reader_status_string(reader_status s) {
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which) {
     if (!ctx || which < 0 || which > 2) return READER_ERR_INVALID_ARG;
     ctx->attn_kernel = which;
+    return READER_OK;
+}
+
+reader_status reader_set_partition(reader_ctx *ctx, int32_t which) {
+    if (!ctx || which < 0 || which > 2) return READER_ERR_INVALID_ARG;
+    ctx->partition = which;
     return READER_OK;
 }
 
@@ -181,6 +189,12 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     p.sched.seq_npages = reinterpret_cast<const int32_t *>(ws + w.seq_npages);
     p.sched.units_per_seq = Hkv;
     p.sched.n_mtiles = n_mtiles;
+    // A shared prefix whose K and V exceed a good part of the L2 is walked by all sequences' lanes in step
+    // (the aligned partition of common.cuh), so that it comes from HBM once; a smaller one stays in L2
+    // whatever the order, and the equal-range partition balances ragged suffixes better.
+    p.sched.aligned = (paged && B >= 2 && (int64_t)p.shared_prefix_pages * Hkv * kPage * D * 2 * 2 > kAlignedPrefixBytes) ? 1 : 0;
+    if (ctx->partition == 1) p.sched.aligned = 0;
+    if (ctx->partition == 2) p.sched.aligned = (paged && B >= 2 && p.shared_prefix_pages > 0) ? 1 : 0;
     PaddedIn pin{};
     reader_kv_cache none{};
     if (padded) {

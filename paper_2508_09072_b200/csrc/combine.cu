@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
     const bool has_cols = lane * 4 < D;
     const int nm = p.sched.n_mtiles;
     const int n_lanes = effective_ctas(p.sched.n_ctas / nm, W);
-    const bool all_live = W >= n_lanes;   // with fewer tiles than CTAs some ranges are empty
+    const bool all_live = !p.sched.aligned && W >= n_lanes;   // with fewer tiles than CTAs some ranges are empty
 
     for (int rb = 0; rb < kRowsPerWarp; rb += kBatch) {
         const int r0 = (blockIdx.y * kCombineWarps + warp) * kRowsPerWarp + rb;
@@ -72,7 +72,11 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 2) combine_kernel(const At
             for (int k = 0; k < 2; ++k) {
                 const int c = cb + k * nm;
                 // a CTA with an empty range wrote nothing
-                const bool live = c <= d.c_last && (all_live || range_begin(c / nm + 1, n_lanes, W) != range_begin(c / nm, n_lanes, W));
+                bool live = c <= d.c_last;
+                if (live && !all_live) {
+                    const LaneRange r = lane_range(p.sched, p.B, c / nm, n_lanes, W);
+                    live = r.w_end > r.w_begin;
+                }
                 const int slot = c == c0 ? 2 * c + 1 : 2 * c;
 #pragma unroll
                 for (int q = 0; q < kBatch; ++q) {

@@ -35,6 +35,7 @@ struct Sched {
     int32_t n_ctas;                 // CTAs launched (n_ctas / n_mtiles lanes); effective_ctas() of the lanes share the work
     int32_t units_per_seq;          // KV streams per sequence: Hkv
     int32_t n_mtiles;               // M tiles per KV stream = CTAs per lane
+    int32_t aligned;                // cut every KV stream at the same relative positions (see lane_range)
 };
 
 struct Segment {
@@ -168,17 +169,84 @@ __device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
     return c;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Aligned partition, for a shared prompt prefix too large to stay in L2 (Sched::aligned).
+//
+// With equal ranges of the flat list the lanes sit at unrelated positions of their KV streams, so the
+// B sequences that share a prefix reach a given prefix tile at B different times and a prefix larger
+// than L2 comes from HBM several times over (measured: 16 sequences over a 134 MB prefix read 1.08 GB).
+// Here every KV stream (sequence b, KV head h) is cut at the same relative positions instead: with at
+// least as many lanes as streams, stream s belongs to the k = n_lanes / n_streams lanes s*k .. s*k+k-1,
+// piece j covering entries [j*len/k, (j+1)*len/k) of it; with fewer lanes, lane l walks the
+// q = ceil(n_streams / n_lanes) whole streams l*q .. l*q+q-1 one after the other.  Either way all lanes
+// start their piece together and advance at the same pace, so the lanes of the sequences sharing a
+// prefix ask for the same prefix tile within a short time of each other: the first fetches it from HBM,
+// the others find it in L2.  The price is load balance (lanes beyond n_streams * k, or the last partial
+// round of streams, idle; streams of different length end at different times), which the equal-range
+// partition does not pay, so it is used only where the prefix would otherwise be re-read.
+// ---------------------------------------------------------------------------------------------
+// First flat entry and number of entries of KV stream `stream` = b * units_per_seq + h.
+__device__ __forceinline__ void stream_span(const Sched &s, int stream, int &start, int &len) {
+    const int b = stream / s.units_per_seq, h = stream - b * s.units_per_seq;
+    const int nt = s.seq_ntiles[b];
+    len = nt > 0 ? nt + kUnitOverhead : 0;
+    start = s.seq_tile_start[b] + h * len;
+}
+
+struct LaneRange {
+    int w_begin, w_end;
+};
+// The range of the flat list that lane `lane` of n_lanes walks; a lane without work gets an empty range.
+__device__ __forceinline__ LaneRange lane_range(const Sched &s, int B, int lane, int n_lanes, int W) {
+    if (!s.aligned) return LaneRange{range_begin(lane, n_lanes, W), range_begin(lane + 1, n_lanes, W)};
+    const int n_streams = B * s.units_per_seq;
+    if (lane >= n_lanes) return LaneRange{W, W};
+    int start, len;
+    if (n_lanes >= n_streams) {
+        const int k = n_lanes / n_streams;
+        const int st = lane / k, j = lane - st * k;
+        if (st >= n_streams) return LaneRange{W, W};
+        stream_span(s, st, start, len);
+        return LaneRange{start + (int)(((int64_t)j * len) / k), start + (int)(((int64_t)(j + 1) * len) / k)};
+    }
+    const int q = (n_streams + n_lanes - 1) / n_lanes;
+    const int s0 = lane * q, s1 = min(n_streams, s0 + q);
+    if (s0 >= n_streams) return LaneRange{W, W};
+    stream_span(s, s0, start, len);
+    int last_start, last_len;
+    stream_span(s, s1 - 1, last_start, last_len);
+    return LaneRange{start, last_start + last_len};
+}
+
+// Lane whose range contains flat entry w, which lies in the unit of segment g (any segment of that unit).
+__device__ __forceinline__ int lane_of_entry(const Sched &s, int B, const Segment &g, int w, int n_lanes, int W) {
+    if (!s.aligned) return cta_of_tile(w, n_lanes, W);
+    const int n_streams = B * s.units_per_seq;
+    const int st = g.b * s.units_per_seq + g.h;
+    if (n_lanes >= n_streams) {
+        const int k = n_lanes / n_streams;
+        const int len = g.ntiles + kUnitOverhead, pos = w - g.unit_w0;
+        int j = (int)(((int64_t)pos * k) / len);
+        if (j >= k) j = k - 1;
+        while (j + 1 < k && (int)(((int64_t)(j + 1) * len) / k) <= pos) ++j;
+        while (j > 0 && (int)(((int64_t)j * len) / k) > pos) --j;
+        return st * k + j;
+    }
+    return st / ((n_streams + n_lanes - 1) / n_lanes);
+}
+
 // The work of one CTA: its M tile and its lane's range of the flat tile list.
 struct CtaWork {
     int mt, n_lanes, w_begin, w_end;
 };
-__device__ __forceinline__ CtaWork cta_work(const Sched &s, int cta, int W) {
+__device__ __forceinline__ CtaWork cta_work(const Sched &s, int B, int cta, int W) {
     CtaWork k;
     const int lane = cta / s.n_mtiles;
     k.mt = cta - lane * s.n_mtiles;
     k.n_lanes = effective_ctas(s.n_ctas / s.n_mtiles, W);   // lanes that share the work
-    k.w_begin = range_begin(lane, k.n_lanes, W);           // a lane left without work gets W, W
-    k.w_end = range_begin(lane + 1, k.n_lanes, W);
+    const LaneRange r = lane_range(s, B, lane, k.n_lanes, W);   // a lane left without work gets an empty range
+    k.w_begin = r.w_begin;
+    k.w_end = r.w_end;
     return k;
 }
 
@@ -190,11 +258,11 @@ struct SplitDesc {
 
 // Called by one thread per segment: if the segment starts its unit without finishing it, note where
 // the unit's partials end so that the combine kernel can find them without any search.
-__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, int n_lanes, const Segment &g, int cta, int W) {
+__device__ __forceinline__ void record_split(SplitDesc *desc, const Sched &s, int B, int n_lanes, const Segment &g, int cta, int W) {
     if (g.tile_begin != 0 || g.full || g.tile_end <= g.tile_begin) return;
     SplitDesc d;
     d.b = g.b; d.h = g.h; d.mt = g.mt;
-    d.c_last = cta_of_tile(g.unit_w0 + kUnitOverhead + g.ntiles - 1, n_lanes, W) * s.n_mtiles + g.mt;   // same M tile, last lane
+    d.c_last = lane_of_entry(s, B, g, g.unit_w0 + kUnitOverhead + g.ntiles - 1, n_lanes, W) * s.n_mtiles + g.mt;   // same M tile, last lane
     desc[cta] = d;
 }
 

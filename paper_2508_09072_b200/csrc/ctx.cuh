@@ -16,6 +16,7 @@ struct reader_ctx {
     int device;
     int n_sm;
     int attn_kernel;  // 0 auto, 1 generic (CUDA cores), 2 tensor-core kernel only
+    int partition;    // 0 auto, 1 equal ranges, 2 aligned whenever a prefix is shared
     reader::Sm100Host sm100;
     cudaEvent_t ev_start, ev_stop;  // optional timing hooks around the main attention kernel
     cudaEvent_t ev_acc_start, ev_acc_stop;  // and around the argmax kernel of reader_accept

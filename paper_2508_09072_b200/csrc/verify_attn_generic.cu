@@ -17,14 +17,14 @@ __global__ void __launch_bounds__(kTileM) attn_generic_kernel(const AttnParams p
     const int cta = blockIdx.x, tid = threadIdx.x;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int W = p.sched.seq_tile_start[p.B];
-    const CtaWork cw = cta_work(p.sched, cta, W);
+    const CtaWork cw = cta_work(p.sched, p.B, cta, W);
     const int w_end = cw.w_end;
     int w = cw.w_begin;
     if (tid == 0) p.split_desc[cta].b = -1;
 
     while (w < w_end) {
         const Segment sg = segment_at(p.sched, p.B, cta, w, w_end);
-        if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
+        if (tid == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
         w += sg.span;
         if (sg.tile_end <= sg.tile_begin) continue;   // the range ended among the unit's overhead entries
 

@@ -5,36 +5,47 @@
 // every unit (sequence, KV head, 128 query rows) a CTA computes S = Q K^T and O += P V with
 // tcgen05.mma, one KV tile of 64 keys (one cache page, or 64 tree nodes) at a time:
 //
-//   warp 4      producer: K tiles and V tiles travel through two separate rings (3 and 2 slots).
+//   warp 8      producer: K tiles and V tiles travel through two separate rings (3 and 2 slots).
 //               Every tile arrives by TMA (64x64 boxes, 128-byte swizzle): cache pages from the
 //               pool (with an L2 evict-first hint when no other CTA will read them again), tree
 //               tiles from the tree tensors, the 128 query rows of the next segment (node j, group
 //               member g -> row j*G+g) by one 4-D box per 64 columns as soon as the previous
 //               segment's last score product is done.  A K slot is free again as soon as its score
 //               product has run, long before the tile's value product, so key loads run far ahead.
-//   warp 5      issues S[i] = Q K[i]^T as soon as K[i] has landed and score buffer i & 1 is free
-//   warp 6      issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Two issuing warps because
+//   warp 9      issues S[i] = Q K[i]^T as soon as K[i] has landed and the score tile is free
+//   warp 10     issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Two issuing warps because
 //               one thread can start a tcgen05.mma only every ~120 cycles: with 8 + 4 of them per
 //               tile a single issuer was the bottleneck of the whole kernel.
-//   warps 0-3   softmax: thread r owns query row r = TMEM lane r.  Scores come from TMEM, the
-//               ancestor bitmask / length mask is applied, the running maximum is raised only
-//               when it grows by more than 2^8 (the accumulator in TMEM is rescaled then),
-//               probabilities (bf16 pairs) are written over the scores they came from and are
-//               the value product's A operand straight from tensor memory.
-//               The same threads write O (or an (m, l, O) partial) at the end of a segment.
+//   warps 0-7   softmax: warp w owns the 16 query rows 32 (w % 4) + 16 (w / 4) .. + 15 (TMEM lanes), a
+//               quad of threads per row pair (rows r and r + 8), so a thread handles 16 of a row's 64
+//               scores and a row's maximum costs two shuffles.  (With one thread per row, 4 warps, a
+//               tile's softmax took ~1350 cycles and sat between the value product of tile i-1 and the
+//               score product of tile i+1 on the critical path; eight warps halve that latency and
+//               give each scheduler four warps to hide it.)  Scores come from TMEM, the ancestor
+//               bitmask / length mask is applied, the running maximum is raised only when it grows
+//               by more than 2^8 (the accumulator in TMEM is rescaled then), probabilities (bf16
+//               pairs) are written over the scores they came from and are the value product's A
+//               operand straight from tensor memory.  The same threads write O (or an (m, l, O)
+//               partial) at the end of a segment.
 //
 // Bytes beyond a sequence's length or the tree's end can never reach a product: scores there are
 // replaced by -inf, and the value product skips 16-key slices past the end and zeroes the tail of
 // the last slice in shared memory first.
 //
-// TMEM: columns 0-127 hold two score buffers of 64 columns (fp32; the first 32 columns of a buffer
-// hold P as bf16 pairs once its softmax is done), columns 128.. hold O (head_dim columns, fp32);
-// lane = query row.
+// TMEM: columns 0-63 hold the score tile S (fp32), columns 64-127 two probability tiles P (32 columns
+// each: bf16 pairs), columns 128.. hold O (head_dim columns, fp32); lane = query row.  S is free again as
+// soon as the softmax warps hold it in registers, so the score product of tile i+1 runs beside the softmax
+// of tile i; P[i & 1] is free once the value product of tile i has read it, two tiles before it is
+// written again.  (With P written over its scores in one of two 64-column buffers, the score product of
+// tile i+1 had to wait for the value product of tile i-1: issue of four value MMAs, issue of eight score
+// MMAs and the softmax sat on one dependency chain per buffer, 1670 cycles per tile of which the tensor
+// pipe worked 45 %.)
 //
-// Barriers: a parity wait can only tell a barrier's current phase from the one before it, so every
-// barrier that warps reach at different times exists once per score buffer; the waiter for tile i on
-// barrier i & 1 knows that tile i-2 is complete and that tile i+2 cannot have been issued.  Every
-// wait is bounded: after one second without progress a CTA raises the error flag in the workspace,
+// Barriers: a parity wait can only tell a barrier's current phase from the one before it.  s_full / s_empty
+// alternate strictly (the score product of tile i+1 needs every softmax thread's arrival for tile i, which
+// comes after that thread saw tile i), so one barrier each is enough; p_full and pv_done, which warps
+// reach at different times, exist once per probability tile: the waiter for tile i on barrier i & 1 knows
+// that tile i-2 is complete and that tile i+2 cannot have been issued.  Every wait is bounded: after one second without progress a CTA raises the error flag in the workspace,
 // stops waiting and runs to its end.
 #include <cuda.h>
 
@@ -50,14 +61,17 @@ using namespace ptx;
 
 constexpr int kStagesK = 3;         // K tiles in flight per CTA (two CTAs share an SM)
 constexpr int kStagesV = 2;         // V tiles
-constexpr int kThreads = 224;
-constexpr int kProducerWarp = 4;
-constexpr int kMmaWarp = 5;   // issues the score products, owns the TMEM allocation
-constexpr int kPvWarp = 6;    // issues the value products
+constexpr int kSoftmaxWarps = 8;   // 16 query rows each
+constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
+constexpr int kProducerWarp = kSoftmaxWarps;
+constexpr int kMmaWarp = kSoftmaxWarps + 1;   // issues the score products, owns the TMEM allocation
+constexpr int kPvWarp = kSoftmaxWarps + 2;    // issues the value products
 constexpr uint64_t kWaitLimitNs = 1000000000ull;
 constexpr float kRaiseMaxBy = 8.f;   // log2 units
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kTmemO = 128;
+constexpr uint32_t kTmemS = 0;      // the score tile (64 columns, fp32)
+constexpr uint32_t kTmemP = 64;     // two probability tiles (32 columns each: bf16 pairs)
+constexpr uint32_t kTmemO = 128;    // the output accumulator (head_dim columns, fp32)
 
 template <int D>
 struct Cfg {
@@ -75,7 +89,7 @@ struct Cfg {
 
 struct Bars {
     uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
-    uint64_t q_full, q_empty, s_full[2], s_empty[2], p_full[2], pv_done[2];
+    uint64_t q_full, q_empty, s_full, s_empty, p_full[2], pv_done[2];
     uint32_t tmem_base;
     int32_t abort;
 };
@@ -240,12 +254,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         }
         mbar_init(bar(&bars->q_full), 1);
         mbar_init(bar(&bars->q_empty), 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(&bars->s_full[s]), 1);
-            mbar_init(bar(&bars->s_empty[s]), 1);
-        }
-        mbar_init(bar(&bars->p_full[0]), kTileM);
-        mbar_init(bar(&bars->p_full[1]), kTileM);
+        mbar_init(bar(&bars->s_full), 1);
+        mbar_init(bar(&bars->s_empty), kSoftmaxWarps * 32);
+        mbar_init(bar(&bars->p_full[0]), kSoftmaxWarps * 32);
+        mbar_init(bar(&bars->p_full[1]), kSoftmaxWarps * 32);
         mbar_init(bar(&bars->pv_done[0]), 1);
         mbar_init(bar(&bars->pv_done[1]), 1);
         bars->abort = 0;
@@ -266,7 +278,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     grid_launch_dependents();
     const WarpSched wsched = load_warp_sched(p.sched, kPadded ? nullptr : p.seq_lens, p.B, lane);   // in flight with W
     const int W = p.sched.seq_tile_start[p.B];
-    const CtaWork cw = cta_work(p.sched, cta, W);
+    const CtaWork cw = cta_work(p.sched, p.B, cta, W);
     const int w_begin = cw.w_begin, w_end = cw.w_end;
 
     if (warp == kProducerWarp) {
@@ -355,10 +367,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (n <= 0) continue;
             wait(bar(&bars->q_full), seg & 1, abort_s, p.error_flag);
             for (int t = 0; t < n; ++t, ++i) {
-                const int stage = i % kStagesK, buf = i & 1;
+                const int stage = i % kStagesK;
                 wait(bar(&bars->k_full[stage]), (i / kStagesK) & 1, abort_s, p.error_flag);
-                // score buffer i & 1 holds P[i-2] until that value product has read it
-                wait(bar(&bars->s_empty[buf]), ((i >> 1) & 1) ^ 1, abort_s, p.error_flag);
+                // the score tile is free as soon as every softmax thread holds the previous scores in registers
+                wait(bar(&bars->s_empty), (i & 1) ^ 1, abort_s, p.error_flag);
                 tc_fence_after();
                 if (lane == 0) {
                     const uint64_t kd = descK + (uint64_t)((stage * C::kTileBytes) >> 4);
@@ -366,10 +378,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                     for (int hf = 0; hf < C::kHalves; ++hf)
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            mma_bf16_ss(tmem + buf * kPage, descQ + (uint64_t)((hf * C::kHalfRowsQ + kk * 32) >> 4),
+                            mma_bf16_ss(tmem + kTmemS, descQ + (uint64_t)((hf * C::kHalfRowsQ + kk * 32) >> 4),
                                         kd + (uint64_t)((hf * C::kHalfRowsKV + kk * 32) >> 4), kIdescQK, (hf | kk) != 0);
                     mma_commit(bar(&bars->k_empty[stage]));
-                    mma_commit(bar(&bars->s_full[buf]));
+                    mma_commit(bar(&bars->s_full));
                     if (t == n - 1) mma_commit(bar(&bars->q_empty));
                 }
                 __syncwarp();
@@ -453,10 +465,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         if (kk < slices)
-                            mma_bf16_ts(tmem + kTmemO, tmem + (i & 1) * kPage + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                            mma_bf16_ts(tmem + kTmemO, tmem + kTmemP + (i & 1) * 32 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
                                         kIdescPV, (tl | kk) != 0);
                     mma_commit(bar(&bars->v_empty[stage]));
-                    mma_commit(bar(&bars->s_empty[i & 1]));
                     mma_commit(bar(&bars->pv_done[i & 1]));
                 }
                 __syncwarp();
@@ -464,118 +475,138 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         }
     } else {
         // ------------------------------------------------------------------ softmax / epilogue
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // this thread: rows row_a and row_b = row_a + 8 of the M tile, columns 8u + 2 cpair (+1), u = 0..7
+        const int cpair = lane & 3;
+        const int row_a = (warp & 3) * 32 + (warp >> 2) * 16 + (lane >> 2), row_b = row_a + 8;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32 + (warp >> 2) * 16) << 16;
+        constexpr uint32_t kNegInf = 0xff800000u;
         int it = 0;
         int w = w_begin;
         if (tid == 0) p.split_desc[cta].b = -1;
         while (w < w_end) {
             const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
-            if (tid == 0) record_split(p.split_desc, p.sched, cw.n_lanes, sg, cta, W);
+            if (tid == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
             w += sg.span;
             if (sg.tile_end <= sg.tile_begin) continue;
             const int L = sg.len;
-            const int grow = sg.mt * kTileM + tid;
-            const bool row_ok = grow < p.T * p.G;
-            const int j = row_ok ? grow / p.G : 0;
-            const int hq = sg.h * p.G + (row_ok ? grow % p.G : 0);
-            const size_t qrow = (((size_t)sg.b * p.T + j) * p.Hq + hq) * D;
+            const int grow_a = sg.mt * kTileM + row_a, grow_b = grow_a + 8;
+            const bool ok_a = grow_a < p.T * p.G, ok_b = grow_b < p.T * p.G;
+            const int j_a = ok_a ? grow_a / p.G : 0, j_b = ok_b ? grow_b / p.G : 0;
+            const int hq_a = sg.h * p.G + (ok_a ? grow_a % p.G : 0), hq_b = sg.h * p.G + (ok_b ? grow_b % p.G : 0);
 
-            uint64_t anc_lo = 0, anc_hi = 0;
-            if (row_ok) {
-                anc_lo = p.anc[((size_t)sg.b * p.T + j) * 2 + 0];
-                anc_hi = p.anc[((size_t)sg.b * p.T + j) * 2 + 1];
+            uint64_t anc_a[2] = {0, 0}, anc_b[2] = {0, 0};
+            if (ok_a) {
+                anc_a[0] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 0];
+                anc_a[1] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 1];
+            }
+            if (ok_b) {
+                anc_b[0] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 0];
+                anc_b[1] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 1];
             }
 
-            float m_used = -INFINITY, l = 0.f;
+            float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // l: this thread's share of the row sums
             for (int t = sg.tile_begin; t < sg.tile_end; ++t, ++it) {
                 // (with a padded cache the mask comes from memory: the load is issued ahead of the wait below)
-                uint64_t vis;
+                uint64_t vis_a, vis_b;
                 if (t < sg.npages) {
-                    vis = visible_of<kPadded>(p, sg.b, t, L);
+                    vis_a = vis_b = visible_of<kPadded>(p, sg.b, t, L);
                 } else {
-                    vis = (t - sg.npages) == 0 ? anc_lo : anc_hi;
+                    vis_a = anc_a[t - sg.npages];
+                    vis_b = anc_b[t - sg.npages];
                 }
                 const int buf = it & 1;
-                wait(bar(&bars->s_full[buf]), (it >> 1) & 1, abort_s, p.error_flag);
+                wait(bar(&bars->s_full), it & 1, abort_s, p.error_flag);
                 tc_fence_after();
-                uint32_t s0[32], s1[32];
-                tmem_ld32(tmem + lane_base + buf * kPage, s0);
-                tmem_ld32(tmem + lane_base + buf * kPage + 32, s1);
+                uint32_t s[32];
+                tmem_ld_16x256b_x8(tmem + lane_base + kTmemS, s);
                 tmem_wait_ld();
+                // the scores are in registers: the next score product may overwrite the tile
+                tc_fence_before();
+                mbar_arrive(bar(&bars->s_empty));
 
-                if (vis != ~0ull) {
-                    const uint32_t lo = (uint32_t)vis, hi = (uint32_t)(vis >> 32);
+                if ((vis_a & vis_b) != ~0ull) {
+                    const uint64_t ma = vis_a >> (2 * cpair), mb = vis_b >> (2 * cpair);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (!((lo >> i) & 1u)) s0[i] = 0xff800000u;
-                        if (!((hi >> i) & 1u)) s1[i] = 0xff800000u;
+                    for (int u = 0; u < 8; ++u) {
+                        if (!((ma >> (8 * u)) & 1ull)) s[4 * u + 0] = kNegInf;
+                        if (!((ma >> (8 * u + 1)) & 1ull)) s[4 * u + 1] = kNegInf;
+                        if (!((mb >> (8 * u)) & 1ull)) s[4 * u + 2] = kNegInf;
+                        if (!((mb >> (8 * u + 1)) & 1ull)) s[4 * u + 3] = kNegInf;
                     }
                 }
-                float mxs[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) mxs[i] = max3(__uint_as_float(s0[i]), __uint_as_float(s1[i]), __uint_as_float(s0[i + 4]));
-#pragma unroll
-                for (int i = 0; i < 4; ++i) mxs[i] = max3(mxs[i], __uint_as_float(s1[i + 4]), __uint_as_float(s0[i + 8]));
-#pragma unroll
-                for (int i = 8; i < 32; i += 8)
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        mxs[q] = max3(mxs[q], __uint_as_float(s1[i + q]), __uint_as_float(s0[i + q + 4]));
-                        mxs[q] = max3(mxs[q], __uint_as_float(s1[i + q + 4]), i + 8 < 32 ? __uint_as_float(s0[i + q + 8]) : -INFINITY);
-                    }
-                const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
-                const float m_new = fmaxf(m_used, mx * p.scale_log2);
+                auto f = [&](int i) { return __uint_as_float(s[i]); };
+                // this thread's 16 scores of each row, then the other three threads of the quad
+                float xa0 = max3(f(0), f(1), f(4)), xa1 = max3(f(5), f(8), f(9));
+                float xb0 = max3(f(2), f(3), f(6)), xb1 = max3(f(7), f(10), f(11));
+                xa0 = max3(xa0, f(12), f(13)); xa1 = max3(xa1, f(16), f(17));
+                xb0 = max3(xb0, f(14), f(15)); xb1 = max3(xb1, f(18), f(19));
+                xa0 = max3(xa0, f(20), f(21)); xa1 = max3(xa1, f(24), f(25));
+                xb0 = max3(xb0, f(22), f(23)); xb1 = max3(xb1, f(26), f(27));
+                float mx_a = max3(xa0, xa1, fmaxf(f(28), f(29))), mx_b = max3(xb0, xb1, fmaxf(f(30), f(31)));
+                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+                const float mn_a = fmaxf(m_a, mx_a * p.scale_log2), mn_b = fmaxf(m_b, mx_b * p.scale_log2);
                 const bool first = t == sg.tile_begin;
-                const bool raise = __any_sync(0xffffffffu, m_new > m_used + kRaiseMaxBy);
-                float alpha = 1.f;
+                const bool raise = __any_sync(0xffffffffu, mn_a > m_a + kRaiseMaxBy || mn_b > m_b + kRaiseMaxBy);
+                float alpha_a = 1.f, alpha_b = 1.f;
                 if (raise || first) {
-                    alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
-                    m_used = m_new;
-                    l *= alpha;
+                    alpha_a = (mn_a == -INFINITY) ? 1.f : ex2(m_a - mn_a);
+                    alpha_b = (mn_b == -INFINITY) ? 1.f : ex2(m_b - mn_b);
+                    m_a = mn_a; m_b = mn_b;
+                    l_a *= alpha_a; l_b *= alpha_b;
                 }
-                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
                 // packed fp32x2 arithmetic: one instruction scales two scores, one adds two probabilities
-                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
-                float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                uint32_t pk[32];
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+                const float nma = (m_a == -INFINITY) ? 0.f : -m_a, nmb = (m_b == -INFINITY) ? 0.f : -m_b;
+                const float2 nma2 = make_float2(nma, nma), nmb2 = make_float2(nmb, nmb);
+                float2 lsa = make_float2(0.f, 0.f), lsb = make_float2(0.f, 0.f);
+                uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s0[2 * i]), __uint_as_float(s0[2 * i + 1])), sc2, nm2);
-                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
-                    ls2[i & 1] = __fadd2_rn(ls2[i & 1], e);
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
-                    pk[i] = *reinterpret_cast<uint32_t *>(&h2);
+                for (int u = 0; u < 8; ++u) {
+                    const float2 xa = __ffma2_rn(make_float2(f(4 * u), f(4 * u + 1)), sc2, nma2);
+                    const float2 xb = __ffma2_rn(make_float2(f(4 * u + 2), f(4 * u + 3)), sc2, nmb2);
+                    const float2 ea = make_float2(ex2(xa.x), ex2(xa.y)), eb = make_float2(ex2(xb.x), ex2(xb.y));
+                    lsa = __fadd2_rn(lsa, ea);
+                    lsb = __fadd2_rn(lsb, eb);
+                    __nv_bfloat162 ha = __floats2bfloat162_rn(ea.x, ea.y), hb = __floats2bfloat162_rn(eb.x, eb.y);
+                    pk[2 * u] = *reinterpret_cast<uint32_t *>(&ha);
+                    pk[2 * u + 1] = *reinterpret_cast<uint32_t *>(&hb);
                 }
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s1[2 * i]), __uint_as_float(s1[2 * i + 1])), sc2, nm2);
-                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
-                    ls2[i & 1] = __fadd2_rn(ls2[i & 1], e);
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
-                    pk[16 + i] = *reinterpret_cast<uint32_t *>(&h2);
-                }
-                l += (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
+                l_a += lsa.x + lsa.y;
+                l_b += lsb.x + lsb.y;
 
                 if (raise && !first) {
                     // O may only be rescaled once the previous value product is complete
                     wait(bar(&bars->pv_done[(it - 1) & 1]), ((it - 1) >> 1) & 1, abort_s, p.error_flag);
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < D; c += 32) {
+                    for (int c = 0; c < D; c += 64) {
                         uint32_t o[32];
-                        tmem_ld32(tmem + lane_base + kTmemO + c, o);
+                        tmem_ld_16x256b_x8(tmem + lane_base + kTmemO + c, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(tmem + lane_base + kTmemO + c, o);
+                        for (int u = 0; u < 8; ++u) {
+                            o[4 * u + 0] = __float_as_uint(__uint_as_float(o[4 * u + 0]) * alpha_a);
+                            o[4 * u + 1] = __float_as_uint(__uint_as_float(o[4 * u + 1]) * alpha_a);
+                            o[4 * u + 2] = __float_as_uint(__uint_as_float(o[4 * u + 2]) * alpha_b);
+                            o[4 * u + 3] = __float_as_uint(__uint_as_float(o[4 * u + 3]) * alpha_b);
+                        }
+                        tmem_st_16x256b_x8(tmem + lane_base + kTmemO + c, o);
                     }
                     tmem_wait_st();
                 }
-                // P (bf16 pairs) replaces the scores it was computed from: 32 columns of this buffer
-                tmem_st32(tmem + lane_base + buf * kPage, pk);
+                // P (bf16 pairs) goes to probability tile it & 1, which the value product of tile it-2 has read by
+                // now; the pair of keys 8u + 2 cpair, + 1 is 32-bit column 4u + cpair
+                if (it >= 2) {
+                    wait(bar(&bars->pv_done[buf]), ((it - 2) >> 1) & 1, abort_s, p.error_flag);
+                    tc_fence_after();
+                }
+                tmem_st_16x128b_x8(tmem + lane_base + kTmemP + buf * 32, pk);
                 tmem_wait_st();
-                // one barrier per score buffer: a warp may be a tile ahead of a slower one (never two,
-                // the next scores for this buffer wait for this tile's value product)
+                // one barrier per probability tile: a warp may be a tile ahead of a slower one (never two: the
+                // store above waits for the value product of tile it-2, which needs every warp's P[it-2])
                 tc_fence_before();
                 mbar_arrive(bar(&bars->p_full[buf]));
             }
@@ -591,45 +622,52 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             // watchdog woke it, about once in a thousand calls.
             wait(bar(&bars->pv_done[(it - 1) & 1]), ((it - 1) >> 1) & 1, abort_s, p.error_flag);
             tc_fence_after();
+            // the row sums: the four shares of the quad
+            l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+            l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+            l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+            l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
             if (sg.full) {
-                const float inv = 1.f / l;   // l > 0 on a valid row: every node sees itself
-                __nv_bfloat16 *dst = p.out + qrow;
+                const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;   // l > 0 on a valid row: every node sees itself
+                __nv_bfloat16 *dst_a = p.out + (((size_t)sg.b * p.T + j_a) * p.Hq + hq_a) * D + 2 * cpair;
+                __nv_bfloat16 *dst_b = p.out + (((size_t)sg.b * p.T + j_b) * p.Hq + hq_b) * D + 2 * cpair;
 #pragma unroll 1
-                for (int c = 0; c < D; c += 32) {
+                for (int c = 0; c < D; c += 64) {
                     uint32_t o[32];
-                    tmem_ld32(tmem + lane_base + kTmemO + c, o);
+                    tmem_ld_16x256b_x8(tmem + lane_base + kTmemO + c, o);
                     tmem_wait_ld();
-                    if (row_ok) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint4 v;
-                            __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                            __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                            __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-                            v.x = *reinterpret_cast<uint32_t *>(&h0);
-                            v.y = *reinterpret_cast<uint32_t *>(&h1);
-                            v.z = *reinterpret_cast<uint32_t *>(&h2);
-                            v.w = *reinterpret_cast<uint32_t *>(&h3);
-                            *reinterpret_cast<uint4 *>(dst + c + 8 * i) = v;
-                        }
+                    for (int u = 0; u < 8; ++u) {
+                        if (ok_a)
+                            *reinterpret_cast<__nv_bfloat162 *>(dst_a + c + 8 * u) =
+                                __floats2bfloat162_rn(__uint_as_float(o[4 * u]) * inv_a, __uint_as_float(o[4 * u + 1]) * inv_a);
+                        if (ok_b)
+                            *reinterpret_cast<__nv_bfloat162 *>(dst_b + c + 8 * u) =
+                                __floats2bfloat162_rn(__uint_as_float(o[4 * u + 2]) * inv_b, __uint_as_float(o[4 * u + 3]) * inv_b);
                     }
                 }
-                if (row_ok && p.lse)
-                    p.lse[((size_t)sg.b * p.T + j) * p.Hq + hq] = (m_used + log2f(l)) * 0.6931471805599453f;
+                if (p.lse && cpair == 0) {
+                    if (ok_a) p.lse[((size_t)sg.b * p.T + j_a) * p.Hq + hq_a] = (m_a + log2f(l_a)) * 0.6931471805599453f;
+                    if (ok_b) p.lse[((size_t)sg.b * p.T + j_b) * p.Hq + hq_b] = (m_b + log2f(l_b)) * 0.6931471805599453f;
+                }
             } else {
-                float *po = p.partial_o + ((size_t)sg.slot * kTileM + tid) * D;
+                float *po_a = p.partial_o + ((size_t)sg.slot * kTileM + row_a) * D + 2 * cpair;
+                float *po_b = p.partial_o + ((size_t)sg.slot * kTileM + row_b) * D + 2 * cpair;
 #pragma unroll 1
-                for (int c = 0; c < D; c += 32) {
+                for (int c = 0; c < D; c += 64) {
                     uint32_t o[32];
-                    tmem_ld32(tmem + lane_base + kTmemO + c, o);
+                    tmem_ld_16x256b_x8(tmem + lane_base + kTmemO + c, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        *reinterpret_cast<uint4 *>(po + c + 4 * i) = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                    for (int u = 0; u < 8; ++u) {
+                        *reinterpret_cast<uint2 *>(po_a + c + 8 * u) = make_uint2(o[4 * u], o[4 * u + 1]);
+                        *reinterpret_cast<uint2 *>(po_b + c + 8 * u) = make_uint2(o[4 * u + 2], o[4 * u + 3]);
+                    }
                 }
-                *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)sg.slot * kTileM + tid) * 2) = make_float2(m_used, l);
-
+                if (cpair == 0) {
+                    *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)sg.slot * kTileM + row_a) * 2) = make_float2(m_a, l_a);
+                    *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)sg.slot * kTileM + row_b) * 2) = make_float2(m_b, l_b);
+                }
             }
             tc_fence_before();
         }

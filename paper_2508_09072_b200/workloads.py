@@ -358,6 +358,21 @@ def make(name: str, with_logits: bool = True, reduced: bool = False, seed_offset
     raise KeyError(name)
 
 
+def make_long_shared_prefix(batch: int = 16, prefix_len: int = 32768, reduced: bool = False) -> Workload:
+    """A shared-prefix batch like C5 whose prefix does not fit the 126 MB L2: `batch` sequences over one
+    prefix of `prefix_len` tokens (16 x 32768: 134 MB of K and V at 8 KV heads, head_dim 128) plus private
+    suffixes of 256..1024 tokens, 32-node trees.  Not one of the five named workloads: it exists to
+    measure how often the attention kernel fetches the prefix from HBM when the cache cannot keep it."""
+    seed = BASE_SEED + 77 + (500 if reduced else 0)
+    rng = np.random.default_rng(seed ^ 0x5EED)
+    if reduced:
+        batch, prefix_len = 3, 512
+    lo, hi = (256, 1024) if not reduced else (40, 150)
+    L = prefix_len + rng.integers(lo, hi + 1, size=batch)
+    return build_workload("long-prefix", seed, L, 32, 32, 8, 128, lambda r: capped_recursive_tree(r, 32, 6, 4),
+                          max_path=6, vocab=16, shuffle_pages=True, shared_prefix_len=prefix_len, with_logits=False)
+
+
 def duplicate_shared_prefix(w: Workload) -> Workload:
     """The same batch with every sequence given private copies of the shared-prefix pages."""
     import copy

@@ -265,6 +265,49 @@ def test_attn_shared_prefix_equals_duplicated_prefix(rd):
     assert err.max() <= 2 ** -6          # the split points differ, so only rounding-level differences
 
 
+ALIGNED_CASES = [
+    # B, Hkv, G, T, D, prefix pages, suffix range: more lanes than KV streams (streams cut in pieces) ...
+    (3, 2, 4, 32, 128, 8, (1, 150)),
+    (2, 1, 8, 64, 128, 20, (0, 70)),        # two M tiles per KV stream
+    (5, 2, 2, 16, 64, 3, (0, 200)),
+    # ... and more KV streams than lanes (whole streams per lane, several rounds)
+    (50, 8, 1, 8, 64, 2, (0, 100)),
+    (41, 8, 4, 32, 128, 1, (1, 64)),
+]
+
+
+@pytest.mark.parametrize("kernel", [2, 1])
+@pytest.mark.parametrize("case", range(len(ALIGNED_CASES)))
+def test_attn_aligned_partition_with_a_shared_prefix(rd, case, kernel):
+    """The partition used for a shared prefix larger than L2 (every KV stream cut at the same relative
+    positions), forced on for shapes the oracle checks in seconds."""
+    B, Hkv, G, T, D, n_prefix, (lo, hi) = ALIGNED_CASES[case]
+    rng = np.random.default_rng(4100 + case)
+    lens = n_prefix * 64 + rng.integers(lo, hi + 1, size=B)
+    w = W.build_workload("al", 4200 + case, lens, T, G * Hkv, Hkv, D, lambda r: W.capped_recursive_tree(r, T, 6, 4),
+                         max_path=6, vocab=16, shuffle_pages=True, shared_prefix_len=n_prefix * 64, with_logits=False)
+    rd.set_partition(2)
+    try:
+        got, status, lse = gpu_attn(rd, w, kernel=kernel)
+    finally:
+        rd.set_partition(0)
+    check_attn(w, got, status, lse)
+    ref, _, _ = gpu_attn(rd, w, kernel=kernel)           # the equal-range partition on the same problem
+    assert np.abs(got - ref).max() <= 2 ** -6
+
+
+def test_attn_shared_prefix_larger_than_l2(rd):
+    """16 sequences over one 32 768-token prefix (134 MB of K and V: more than the L2 holds) plus private
+    suffixes: every element against the oracle, and against the same batch with the prefix stored once
+    per sequence (which takes the equal-range partition)."""
+    w = W.make_long_shared_prefix()
+    got, status, lse = gpu_attn(rd, w, kernel=2)
+    assert not status.any()
+    check_attn(w, got, status, lse)
+    dup, _, _ = gpu_attn(rd, W.duplicate_shared_prefix(w), kernel=2)
+    assert np.abs(got - dup).max() <= 2 ** -6
+
+
 @pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
 def test_attn_full_size_every_element_against_oracle(rd, name):
     """Full workload sizes in the launch configuration the benchmark times, on the tensor-core kernel
