@@ -538,17 +538,34 @@ void oracle_sample_targets(const float *logits, const int32_t *parent, const flo
                            int B, int T, int64_t vocab, double temperature, int64_t top_k, float top_p,
                            int32_t *target)
 {
+    /* One uniform per output position (Appendix C): position = tree level, taken from
+     * oracle_levels, the same function the attention pins use.  Only for a parent
+     * array that is not a tree (no level exists) is a position made up, by counting
+     * the nodes met while the parent index keeps decreasing, so that any input gives
+     * a defined result. */
+    int32_t *level = (int32_t *)malloc(sizeof(int32_t) * (size_t)B * T);
+    if (!level) return;
+    for (int b = 0; b < B; ++b) {
+        const int32_t *par = parent + (size_t)b * T;
+        if (oracle_tree_is_valid(par, T)) {
+            oracle_levels(par, T, level + (size_t)b * T);
+            continue;
+        }
+        for (int j = 0; j < T; ++j) {
+            int count = 0;
+            for (int i = j, steps = 0; i >= 0 && i < T && steps < T; ++steps) {
+                ++count;
+                i = par[i] < i ? par[i] : -1;
+            }
+            level[(size_t)b * T + j] = count;
+        }
+    }
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < (int64_t)B * T; ++r) {
-        const int b = (int)(r / T), j = (int)(r % T);
-        int lv = 0;
-        for (int i = j, steps = 0; i >= 0 && i < T && steps < T; ++steps) {
-            ++lv;
-            const int up = parent[(size_t)b * T + i];
-            i = up < i ? up : -1;                 /* a malformed array cannot send the walk astray */
-        }
-        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + lv - 1], temperature, top_k, top_p);
+        const int b = (int)(r / T);
+        target[r] = oracle_sample_row(logits + r * vocab, vocab, uniforms[(size_t)b * T + level[r] - 1], temperature, top_k, top_p);
     }
+    free(level);
 }
 
 void oracle_accept(const int32_t *parent, const int32_t *tok, const int32_t *target,

@@ -162,3 +162,54 @@ def test_randomized_losslessness_with_coupled_uniforms():
         n_steps += 1
     assert out[: steps + 1] == base[: steps + 1]
     assert n_steps < steps                                       # several tokens per step were accepted
+
+
+def _exact_cdf(logits, temperature, top_k, top_p):
+    """Plain fp64 statement of F (Appendix C): temperature softmax, top-k by value (ties kept), then the
+    smallest set of highest logits whose mass reaches top_p (ties kept); returns the inclusive CDF over
+    token ids, the kept mask and how close the nucleus came to its threshold."""
+    z = logits.astype(np.float64) / temperature
+    keep = np.ones(len(z), bool)
+    if top_k > 0 and top_k < len(z):
+        kth = np.sort(z)[::-1][top_k - 1]
+        keep &= z >= kth
+    w = np.where(keep, np.exp(z - z[keep].max()), 0.0)
+    margin = np.inf
+    if top_p < 1.0:
+        order = np.argsort(-z, kind="stable")
+        order = order[keep[order]]
+        mass = np.cumsum(w[order]) / w.sum()
+        first = int(np.argmax(mass >= top_p))               # last admitted rank
+        cut = z[order[first]]
+        margin = min(abs(mass[first] - top_p), abs(mass[first - 1] - top_p) if first > 0 else np.inf)
+        keep &= z >= cut
+        w = np.where(keep, w, 0.0)
+    return np.cumsum(w) / w.sum(), keep, margin
+
+
+@pytest.mark.parametrize("top_k,top_p", [(0, 1.0), (7, 1.0), (0, 0.8), (40, 0.6)])
+def test_choice_agrees_with_the_plain_fp64_inverse_cdf(top_k, top_p):
+    """The integer recipe (a polynomial for 2^f, 40-bit weights, a 24-bit uniform) is this library's own; what
+    it must realise is x* = F(P, u) for the plain softmax CDF.  For random rows and uniforms the token it
+    picks is the one the fp64 CDF picks, except where u lies within 3e-5 of a CDF step (the recipe's stated
+    accuracy: 2^f to 3e-6, u to 2^-24)."""
+    rng = np.random.default_rng(100 + top_k)
+    eps, off = 3e-5, 0
+    for trial in range(24):
+        V = int(rng.choice([17, 64, 300, 2000]))
+        temperature = float(rng.choice([0.5, 1.0, 1.7]))
+        lg = (rng.standard_normal(V) * rng.choice([0.5, 2.0, 5.0])).astype(np.float32)
+        cdf, keep, margin = _exact_cdf(lg, temperature, top_k, top_p)
+        if margin < 1e-4:
+            continue                                        # the nucleus itself hinges on rounding: not a case for this pin
+        us = rng.random(300).astype(np.float32)
+        got = oracle.sample_targets(np.tile(lg, (len(us), 1, 1)), np.full((len(us), 1), -1, np.int32), us.reshape(-1, 1),
+                                    temperature, top_k, top_p)[:, 0]
+        want = np.searchsorted(cdf, us.astype(np.float64), side="right")
+        for u, g, x in zip(us.astype(np.float64), got, want):
+            assert keep[g], (trial, u, g)                   # never a filtered token
+            if g != x:
+                lo = cdf[g - 1] if g > 0 else 0.0
+                assert lo - eps <= u <= cdf[g] + eps, (trial, V, temperature, u, g, x)
+                off += 1
+    assert off <= 5                                         # boundary cases are rare
