@@ -114,10 +114,12 @@ reader_status reader_create(reader_ctx **out, int device);
 void reader_destroy(reader_ctx *ctx);
 const char *reader_status_string(reader_status s);
 
-/* Chooses the attention kernel: 0 = automatic (the tensor-core kernel; the CUDA-core kernel only for
- * the shapes the former is not built for: a GQA group that does not divide 128, a non-positive
- * scale), 1 = always the CUDA-core kernel, 2 = tensor-core kernel or READER_ERR_UNSUPPORTED.
- * Both compute Sec. 3.2's attention; this is a testing aid. Host call. */
+/* Chooses the attention kernel: 0 = automatic (the tensor-core kernel, as a single launch for calls with
+ * few units and as preparation + attention + combine otherwise; the CUDA-core kernel only for the shapes
+ * the former is not built for: a GQA group that does not divide 128, a non-positive scale), 1 = always
+ * the CUDA-core kernel, 2 = the tensor-core kernel on the three-launch path or READER_ERR_UNSUPPORTED,
+ * 3 = the tensor-core kernel as a single launch or READER_ERR_UNSUPPORTED (batch * n_kv_heads * M tiles
+ * must fit the GPU in one wave).  All compute Sec. 3.2's attention; this is a testing aid. Host call. */
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which);
 
 /* Chooses how reader_verify_attn divides its work among thread blocks: 0 = automatic, 1 = always equal

@@ -12,6 +12,7 @@ namespace {
 using namespace reader;
 
 constexpr int kMaxSplits = kMaxArgmaxSplits;
+constexpr int kSmallTilesPerCta = 12;   // largest share of a unit that still counts as a small call
 constexpr int64_t kAlignedPrefixBytes = 48ll << 20;   // shared prefix K+V above which the lanes walk it in step (L2: 126 MB)
 constexpr size_t kAlign = 256;
 
@@ -110,7 +111,7 @@ const char *reader_status_string(reader_status s) {
 }
 
 reader_status reader_set_attn_kernel(reader_ctx *ctx, int32_t which) {
-    if (!ctx || which < 0 || which > 2) return READER_ERR_INVALID_ARG;
+    if (!ctx || which < 0 || which > 3) return READER_ERR_INVALID_ARG;
     ctx->attn_kernel = which;
     return READER_OK;
 }
@@ -209,8 +210,25 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     }
 
     const bool tc_ok = sm100_supports(&ctx->sm100, p, softmax_scale);
-    if (ctx->attn_kernel == 2 && !tc_ok && mode != kPrepareOnly) return READER_ERR_UNSUPPORTED;
+    if (ctx->attn_kernel >= 2 && !tc_ok && mode != kPrepareOnly) return READER_ERR_UNSUPPORTED;
     const bool use_tc = tc_ok && ctx->attn_kernel != 1;
+    // A call with few units (one or a few sequences: the batch-1 regime of Sec. 4.1) is three dependent
+    // launches of mostly latency on the general path.  It takes one launch instead: every unit
+    // (sequence, KV head, M tile) gets a cluster of up to 8 CTAs that checks the sequence, shares the unit's
+    // tiles and merges the shares in distributed shared memory.  Chosen when the clusters fit the GPU in one
+    // wave and a share is at most kSmallTilesPerCta tiles (judged by the page table's width: lengths live on
+    // the device); reader_set_attn_kernel(3) takes it whenever the clusters fit.
+    int small_cluster = 0;
+    p.parent = tree->parent;
+    if (use_tc && paged && !p.sched.aligned && ctx->attn_kernel != 2) {
+        const int64_t n_units = (int64_t)B * Hkv * n_mtiles, bound = max_pages + n_tree_tiles;
+        int cs = 8;
+        while (cs > 1 && (bound < 2 * cs || n_units * cs > max_ctas(ctx))) cs >>= 1;
+        const bool fits = n_units * cs <= max_ctas(ctx);
+        if (fits && (ctx->attn_kernel == 3 || (bound + cs - 1) / cs <= kSmallTilesPerCta)) small_cluster = cs;
+    }
+    if (ctx->attn_kernel == 3 && small_cluster == 0 && mode != kPrepareOnly) return READER_ERR_UNSUPPORTED;
+    if (small_cluster > 0 && mode == kPrepareAndRun && !tree->anc_mask) p.anc = nullptr;   // no preparation runs: masks from the parent array
     // Two resident CTAs per SM for both kernels -- fewer when the page table is too narrow to give that many
     // CTAs work: on the device effective_ctas() never uses more than ceil(W / kMinTilesPerCta) lanes, and W
     // cannot exceed the bound below, so the partition is the same and the launches are smaller.
@@ -221,7 +239,7 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
         p.sched.n_ctas = (int)(busy < max_ctas(ctx) ? busy : max_ctas(ctx));
     }
 
-    if (mode != kRunPrepared)
+    if (mode == kPrepareOnly || (mode == kPrepareAndRun && small_cluster == 0))
         launch_prepare(paged ? *paged : none, pin, tree->parent, B, T, n_tree_tiles, p.sched.units_per_seq,
                    tree->anc_mask ? nullptr : reinterpret_cast<uint64_t *>(ws + w.anc),
                    reinterpret_cast<int32_t *>(ws + w.seq_tile_start), reinterpret_cast<int32_t *>(ws + w.seq_ntiles),
@@ -229,12 +247,12 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     if (mode == kPrepareOnly) return launch_status();
     if (ctx->ev_start) cudaEventRecord(ctx->ev_start, st);
     if (use_tc) {
-        if (reader_status s = launch_attn_sm100(&ctx->sm100, p, st)) return s;
+        if (reader_status s = launch_attn_sm100(&ctx->sm100, p, small_cluster, st)) return s;
     } else {
         launch_attn_generic(p, st);
     }
     if (ctx->ev_stop) cudaEventRecord(ctx->ev_stop, st);
-    launch_combine(p, st);
+    if (small_cluster == 0) launch_combine(p, st);
     return launch_status();
 }
 

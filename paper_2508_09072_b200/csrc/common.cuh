@@ -294,6 +294,7 @@ struct AttnParams {
     int bits_per_seq, cap;
     int zero_rejected;         // the combine kernel zeroes the rows of sequences whose status word is set (the
                                // preparation ran in an earlier call and could not know this call's output)
+    const int32_t *parent;     // [B][T] (the single-launch kernel for small calls checks the trees itself)
     Sched sched;
 };
 

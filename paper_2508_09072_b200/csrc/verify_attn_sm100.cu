@@ -52,6 +52,7 @@
 #include <new>
 
 #include "ptx_sm100.cuh"
+#include "tree.cuh"
 #include "verify_attn_sm100.cuh"
 
 namespace reader {
@@ -85,6 +86,9 @@ struct Cfg {
     static constexpr int kOffV = kOffK + kStagesK * kTileBytes;    // ring of V tiles
     static constexpr int kOffBars = kOffV + kStagesV * kTileBytes;
     static constexpr int kSmemBytes = kOffBars + 256;   // + barriers; two CTAs of head_dim 128 fit one SM
+    // the single-launch kernel for small calls also keeps one sequence's parent array there
+    static constexpr int kOffParents = kOffBars + 256;
+    static constexpr int kSmemBytesSmall = kOffParents + kMaxNodes * 4;
 };
 
 struct Bars {
@@ -92,6 +96,7 @@ struct Bars {
     uint64_t q_full, q_empty, s_full, s_empty, p_full[2], pv_done[2];
     uint32_t tmem_base;
     int32_t abort;
+    int32_t reject;   // small-call kernel: status code of a sequence the checks turned down
 };
 static_assert(sizeof(Bars) <= 256, "barrier block");
 
@@ -150,12 +155,28 @@ __device__ __forceinline__ uint64_t visible_of(const AttnParams &p, int b, int t
     }
 }
 
+// Where a CTA's work comes from.  The general kernel walks a range of the flattened tile list laid out by
+// the preparation kernel; the single-launch kernel for small calls (kSmall) has exactly one segment, the
+// share of its unit's tiles that its rank in the cluster gives it, and counts flat positions in tiles.
+template <bool kSmall, bool kPadded>
+__device__ __forceinline__ Segment seg_at(const AttnParams &p, const WarpSched &ws, const Segment &mine, int cta, int w, int w_end,
+                                          int lane) {
+    if constexpr (kSmall) {
+        Segment g = mine;
+        g.tile_begin = mine.tile_begin + w;
+        g.span = w_end - w;
+        return g;
+    } else {
+        return segment_at_warp(p.sched, ws, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
+    }
+}
+
 // Walks the tiles of a CTA's range in order; the producer keeps one cursor for keys and one for
 // values.  Page ids are fetched 32 at a time (one per lane) and handed out by shuffle.
-template <bool kPadded>
+template <bool kPadded, bool kSmall>
 struct TileCursor {
     int w, w_end;       // flat position of the next segment
-    Segment sg;
+    Segment sg, mine;
     int L;              // committed length of sg.b
     int t;              // current tile within the unit
     int it;             // tiles handed out so far
@@ -171,7 +192,7 @@ struct TileCursor {
     __device__ __forceinline__ void next_segment(const AttnParams &p, const WarpSched &ws, int cta, int lane) {
         active = false;
         while (w < w_end) {   // segments without a real tile (a range that ends among overhead entries) are skipped
-            sg = segment_at_warp(p.sched, ws, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
+            sg = seg_at<kSmall, kPadded>(p, ws, mine, cta, w, w_end, lane);
             w += sg.span;
             if (sg.tile_end > sg.tile_begin) { active = true; break; }
         }
@@ -180,7 +201,9 @@ struct TileCursor {
         t = sg.tile_begin;
         refill(p, lane);
     }
-    __device__ __forceinline__ void init(const AttnParams &p, const WarpSched &ws, int cta, int lane, int w_begin, int w_end_) {
+    __device__ __forceinline__ void init(const AttnParams &p, const WarpSched &ws, const Segment &mine_, int cta, int lane, int w_begin,
+                                         int w_end_) {
+        mine = mine_;
         w = w_begin; w_end = w_end_; it = 0;
         next_segment(p, ws, cta, lane);
     }
@@ -197,8 +220,8 @@ struct TileCursor {
 // one KV head from the tree tensor (rows past the tensor's end read as zero).  Rows past the
 // valid count may therefore hold anything; the score side masks them by selection and the value
 // side never multiplies them (see the MMA issuer).  Called by the whole producer warp.
-template <int D, bool kPadded>
-__device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor<kPadded> &c, const CUtensorMap *pool_map,
+template <int D, bool kPadded, bool kSmall>
+__device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor<kPadded, kSmall> &c, const CUtensorMap *pool_map,
                                           const CUtensorMap *tree_map, uint32_t dst, uint32_t full, int lane,
                                           uint64_t stream_policy, int first_streamed_tile) {
     using C = Cfg<D>;
@@ -222,7 +245,7 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor<
     }
 }
 
-template <int D, bool kPadded>
+template <int D, bool kPadded, bool kSmall>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                   const __grid_constant__ CUtensorMap ktmap, const __grid_constant__ CUtensorMap vtmap,
@@ -261,6 +284,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         mbar_init(bar(&bars->pv_done[0]), 1);
         mbar_init(bar(&bars->pv_done[1]), 1);
         bars->abort = 0;
+        bars->reject = 0;
         fence_mbar_init();
         fence_proxy_async();
     }
@@ -273,13 +297,55 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
-    // everything above overlapped the preparation kernel; its results are read from here on
+    // everything above overlapped the kernel before this one in the stream; its results are read from here on
     grid_dependency_wait();
     grid_launch_dependents();
-    const WarpSched wsched = load_warp_sched(p.sched, kPadded ? nullptr : p.seq_lens, p.B, lane);   // in flight with W
-    const int W = p.sched.seq_tile_start[p.B];
-    const CtaWork cw = cta_work(p.sched, p.B, cta, W);
-    const int w_begin = cw.w_begin, w_end = cw.w_end;
+    WarpSched wsched{0x7fffffff, 0, 0, 0};
+    CtaWork cw{0, 0, 0, 0};
+    Segment mine{};          // kSmall: this CTA's share of its unit
+    int W = 0, w_begin = 0, w_end = 0;
+    int reject = 0;          // kSmall: status code of a sequence the checks below turn down
+    uint32_t cl_rank = 0, cl_size = 1;
+    const int32_t *par = reinterpret_cast<const int32_t *>(smem + C::kOffParents);   // kSmall only
+    if constexpr (kSmall) {
+        // One launch does everything for a call with few units: the cluster (b, KV head, M tile) checks its
+        // sequence itself (what the preparation kernel does for large calls), cuts the unit's tiles into one
+        // share per CTA of the cluster, and merges the shares (partials in the workspace, ordered by the
+        // cluster's hardware barrier) at the end.
+        cl_rank = cluster_ctarank();
+        cl_size = cluster_nctarank();
+        const int n_mtiles = (p.T * p.G + kTileM - 1) / kTileM;
+        const int unit = cta / (int)cl_size;
+        mine.mt = unit % n_mtiles;
+        mine.h = (unit / n_mtiles) % p.Hkv;
+        mine.b = unit / (n_mtiles * p.Hkv);
+        // Only the committed length is needed to start loading: the checks of the tree and of the page ids run
+        // in the softmax warps (below) while the first tiles are on their way, and their verdict is used at the
+        // end.  (A page id outside the pool makes a tile load read the fill value, never a fault.)
+        const int L = p.seq_lens[mine.b];
+        const bool len_ok = L >= 0 && (int64_t)L <= (int64_t)p.max_pages * kPage;
+        const bool flagged = p.zero_rejected && *p.error_flag != 0;   // a layer call after a layer that gave up a wait
+        const int npages = (len_ok && !flagged) ? (L + kPage - 1) / kPage : 0;
+        const int n = (len_ok && !flagged) ? npages + (p.T + kPage - 1) / kPage : 0;
+        mine.ntiles = n;
+        mine.npages = npages;
+        mine.len = L;
+        mine.tile_begin = (int)(((int64_t)cl_rank * n) / cl_size);
+        mine.tile_end = (int)(((int64_t)(cl_rank + 1) * n) / cl_size);
+        mine.full = cl_size == 1;
+        mine.slot = cta;
+        w_end = mine.tile_end - mine.tile_begin;
+        if (tid == 0) {
+            if (flagged) atomicOr(&bars->reject, 8);
+            else if (!len_ok) atomicOr(&bars->reject, 2);
+        }
+    } else {
+        wsched = load_warp_sched(p.sched, kPadded ? nullptr : p.seq_lens, p.B, lane);   // in flight with W
+        W = p.sched.seq_tile_start[p.B];
+        cw = cta_work(p.sched, p.B, cta, W);
+        w_begin = cw.w_begin;
+        w_end = cw.w_end;
+    }
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
@@ -294,9 +360,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         // shared prefix the hint measured slightly slower, so it is left off there)
         const uint64_t stream_policy = l2_policy_evict_first();
         const int first_streamed_tile = (p.sched.n_mtiles == 1 && p.shared_prefix_pages == 0) ? 0 : 0x7fffffff;
-        TileCursor<kPadded> kc, vc;
-        kc.init(p, wsched, cta, lane, w_begin, w_end);
-        vc.init(p, wsched, cta, lane, w_begin, w_end);
+        TileCursor<kPadded, kSmall> kc, vc;
+        kc.init(p, wsched, mine, cta, lane, w_begin, w_end);
+        vc.init(p, wsched, mine, cta, lane, w_begin, w_end);
         // the query tile of the next segment goes in as soon as the last score product of the
         // current one has retired (Q is single-buffered)
         int q_w = w_begin, q_seg = 0;
@@ -305,7 +371,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         while (kc.active || vc.active || q_w < w_end) {
             bool moved = false;
             if (q_w < w_end && ready(bar(&bars->q_empty), (q_seg & 1) ^ 1)) {
-                const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, q_w, w_end, lane);
+                const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, q_w, w_end, lane);
                 q_w += sg.span;
                 if (sg.tile_end <= sg.tile_begin) continue;   // no real tile: no query tile
                 if (lane == 0) {
@@ -322,7 +388,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (kc.active) {
                 const int stage = kc.it % kStagesK;
                 if (ready(bar(&bars->k_empty[stage]), ((kc.it / kStagesK) & 1) ^ 1)) {
-                    load_tile<D, kPadded>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
+                    load_tile<D, kPadded, kSmall>(p, kc, &kmap, &ktmap, sK + stage * C::kTileBytes, bar(&bars->k_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     kc.advance(p, wsched, cta, lane);
                     moved = true;
@@ -331,7 +397,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             if (vc.active) {
                 const int stage = vc.it % kStagesV;
                 if (ready(bar(&bars->v_empty[stage]), ((vc.it / kStagesV) & 1) ^ 1)) {
-                    load_tile<D, kPadded>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
+                    load_tile<D, kPadded, kSmall>(p, vc, &vmap, &vtmap, sV + stage * C::kTileBytes, bar(&bars->v_full[stage]), lane, stream_policy, first_streamed_tile);
                     __syncwarp();
                     vc.advance(p, wsched, cta, lane);
                     moved = true;
@@ -361,7 +427,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int i = 0, seg = 0;
         int w = w_begin;
         while (w < w_end && !*abort_s) {
-            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
+            const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += sg.span;
             if (n <= 0) continue;
@@ -395,7 +461,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         int i = 0;
         int w = w_begin;
         while (w < w_end && !*abort_s) {
-            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
+            const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
             w += sg.span;
             if (n <= 0) continue;
@@ -473,7 +539,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 __syncwarp();
             }
         }
-    } else {
+    } else if (warp < kSoftmaxWarps) {
         // ------------------------------------------------------------------ softmax / epilogue
         // this thread: rows row_a and row_b = row_a + 8 of the M tile, columns 8u + 2 cpair (+1), u = 0..7
         const int cpair = lane & 3;
@@ -482,10 +548,37 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         constexpr uint32_t kNegInf = 0xff800000u;
         int it = 0;
         int w = w_begin;
-        if (tid == 0) p.split_desc[cta].b = -1;
+        bool tree_ok = true;
+        if constexpr (kSmall) {
+            // the checks the preparation kernel makes for large calls: parent[0] = -1 and 0 <= parent[j] < j; every
+            // page id in use inside the pool.  256 threads, then one barrier among the softmax warps.
+            int32_t *par_w = reinterpret_cast<int32_t *>(smem + C::kOffParents);
+            int bits = 0;
+            for (int j = tid; j < p.T; j += kSoftmaxWarps * 32) {
+                const int pj = p.parent[(size_t)mine.b * p.T + j];
+                par_w[j] = pj;
+                if (!(j == 0 ? pj == -1 : (pj >= 0 && pj < j))) bits |= 1;
+            }
+            for (int i = tid; i < mine.npages; i += kSoftmaxWarps * 32) {
+                const int pg = p.page_table[(size_t)mine.b * p.max_pages + i];
+                if (pg < 0 || pg >= p.num_pages) bits |= 4;
+            }
+            if (bits) atomicOr(&bars->reject, bits);
+            asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxWarps * 32) : "memory");
+            tree_ok = (*reinterpret_cast<volatile int32_t *>(&bars->reject) & 1) == 0;
+        }
+        if constexpr (!kSmall) {
+            if (tid == 0) p.split_desc[cta].b = -1;
+        } else if (w_end == 0 && cpair == 0) {
+            // no tile fell to this CTA: its share of the unit is the empty partial
+            *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)cta * kTileM + row_a) * 2) = make_float2(-INFINITY, 0.f);
+            *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)cta * kTileM + row_b) * 2) = make_float2(-INFINITY, 0.f);
+        }
         while (w < w_end) {
-            const Segment sg = segment_at_warp(p.sched, wsched, kPadded ? nullptr : p.seq_lens, p.B, cta, w, w_end, lane);
-            if (tid == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
+            const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, w, w_end, lane);
+            if constexpr (!kSmall) {
+                if (tid == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
+            }
             w += sg.span;
             if (sg.tile_end <= sg.tile_begin) continue;
             const int L = sg.len;
@@ -495,13 +588,19 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             const int hq_a = sg.h * p.G + (ok_a ? grow_a % p.G : 0), hq_b = sg.h * p.G + (ok_b ? grow_b % p.G : 0);
 
             uint64_t anc_a[2] = {0, 0}, anc_b[2] = {0, 0};
-            if (ok_a) {
-                anc_a[0] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 0];
-                anc_a[1] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 1];
-            }
-            if (ok_b) {
-                anc_b[0] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 0];
-                anc_b[1] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 1];
+            if (kSmall && p.anc == nullptr) {   // no encoded masks at hand: walk the parent array (in shared memory)
+                int lv;
+                if (ok_a && tree_ok) node_ancestors(par, p.T, j_a, anc_a[0], anc_a[1], lv);
+                if (ok_b && tree_ok) node_ancestors(par, p.T, j_b, anc_b[0], anc_b[1], lv);
+            } else {
+                if (ok_a) {
+                    anc_a[0] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 0];
+                    anc_a[1] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 1];
+                }
+                if (ok_b) {
+                    anc_b[0] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 0];
+                    anc_b[1] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 1];
+                }
             }
 
             float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // l: this thread's share of the row sums
@@ -651,6 +750,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                     if (ok_b) p.lse[((size_t)sg.b * p.T + j_b) * p.Hq + hq_b] = (m_b + log2f(l_b)) * 0.6931471805599453f;
                 }
             } else {
+                // (single-launch kernel: slot = this CTA; the cluster's CTAs fetch the rows they merge from there)
                 float *po_a = p.partial_o + ((size_t)sg.slot * kTileM + row_a) * D + 2 * cpair;
                 float *po_b = p.partial_o + ((size_t)sg.slot * kTileM + row_b) * D + 2 * cpair;
 #pragma unroll 1
@@ -675,6 +775,83 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (kSmall) {
+        // The shares of a unit meet here: CTA r of the cluster merges rows 128 r / size .. of the unit out of
+        // every CTA's partial (m* = max m_s, l* = sum l_s 2^(m_s - m*), O = sum O_s 2^(m_s - m*) / l*)
+        // and writes them.  A rejected sequence, or a CTA that gave up on a bounded wait, gets zero rows.
+        const bool multi = cl_size > 1;
+        const int rb = bars->reject;   // complete: every warp has passed the barrier above
+        reject = (rb & 8) ? *p.error_flag : (rb & 1) ? READER_ERR_BAD_TREE : (rb & 2) ? READER_ERR_CAPACITY : (rb & 4) ? READER_ERR_BAD_PAGE : 0;
+        if (tid == 0 && cl_rank == 0 && mine.h == 0 && mine.mt == 0) p.status[mine.b] = reject;
+        const bool gave_up = *abort_s != 0;
+        if (multi) {
+            if (tid == 0) p.split_desc[cta].b = gave_up ? 1 : 0;   // this CTA's give-up flag, beside its partial
+            cluster_arrive_release();
+            cluster_wait_acquire();
+        }
+        if (warp < kSoftmaxWarps && (multi || reject != 0 || gave_up)) {
+            const int rows_per = kTileM / (int)cl_size;
+            const bool has_cols = lane * 4 < D;
+            const int cta0 = cta - (int)cl_rank;   // the cluster's first CTA: share q lies in partial slot cta0 + q
+            int peer_flag = 0;   // consumed after the first row's loads have been issued: one round trip to L2, not two
+            if (multi && lane < (int)cl_size) peer_flag = __ldcg(&p.split_desc[cta0 + lane].b);
+            bool peer_gave_up = false, flags_read = false;
+            for (int rr = warp; rr < rows_per; rr += kSoftmaxWarps) {
+                const int row = (int)cl_rank * rows_per + rr;
+                const int grow = mine.mt * kTileM + row;
+                if (grow >= p.T * p.G) continue;
+                float mstar = -INFINITY, lstar = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                bool bad = reject != 0 || gave_up;
+                if (multi && reject == 0) {
+                    // every share's row in flight at once.  The shares travel through the workspace (L2), not through
+                    // distributed shared memory: reads of another CTA's shared memory came back one at a time,
+                    // 0.3 us each, which made this merge 5 us long on eight shares.
+                    constexpr int kMaxCluster = 8;
+                    float2 ml[kMaxCluster];
+                    float4 o[kMaxCluster];
+#pragma unroll
+                    for (int q = 0; q < kMaxCluster; ++q) {
+                        ml[q] = make_float2(-INFINITY, 0.f);
+                        o[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (q < (int)cl_size) {
+                            ml[q] = __ldcg(reinterpret_cast<const float2 *>(p.partial_ml + ((size_t)(cta0 + q) * kTileM + row) * 2));
+                            if (has_cols) o[q] = __ldcg(reinterpret_cast<const float4 *>(p.partial_o + ((size_t)(cta0 + q) * kTileM + row) * D + lane * 4));
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < kMaxCluster; ++q) mstar = fmaxf(mstar, ml[q].x);
+                    if (!flags_read) {
+                        peer_gave_up = __any_sync(0xffffffffu, peer_flag != 0);
+                        flags_read = true;
+                    }
+                    bad = bad || peer_gave_up;
+#pragma unroll
+                    for (int q = 0; q < kMaxCluster; ++q) {
+                        const float wgt = ml[q].x == -INFINITY ? 0.f : exp2f(ml[q].x - mstar);   // an empty share holds no row
+                        lstar = fmaf(ml[q].y, wgt, lstar);
+                        acc.x = fmaf(wgt == 0.f ? 0.f : o[q].x, wgt, acc.x);
+                        acc.y = fmaf(wgt == 0.f ? 0.f : o[q].y, wgt, acc.y);
+                        acc.z = fmaf(wgt == 0.f ? 0.f : o[q].z, wgt, acc.z);
+                        acc.w = fmaf(wgt == 0.f ? 0.f : o[q].w, wgt, acc.w);
+                    }
+                }
+                const int j = grow / p.G, hq = mine.h * p.G + grow % p.G;
+                const size_t orow = ((size_t)mine.b * p.T + j) * p.Hq + hq;
+                const float inv = bad ? 0.f : 1.f / lstar;
+                if (has_cols) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(bad ? 0.f : acc.x * inv, bad ? 0.f : acc.y * inv);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(bad ? 0.f : acc.z * inv, bad ? 0.f : acc.w * inv);
+                    uint2 v;
+                    v.x = *reinterpret_cast<uint32_t *>(&lo);
+                    v.y = *reinterpret_cast<uint32_t *>(&hi);
+                    *reinterpret_cast<uint2 *>(p.out + orow * D + lane * 4) = v;
+                }
+                if (p.lse && lane == 0) p.lse[orow] = bad ? 0.f : (mstar + log2f(lstar)) * 0.6931471805599453f;
+                if (bad && reject == 0 && lane == 0) atomicMax(&p.status[mine.b], (int32_t)READER_ERR_TIMEOUT);
+            }
+        }
+    }
     if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
@@ -787,12 +964,16 @@ bool sm100_supports(const Sm100Host *h, const AttnParams &p, float softmax_scale
     return (p.D == 64 || p.D == 128) && rows >= 1 && rows < ((int64_t)1 << 31);
 }
 
-reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t st) {
+// small_cluster = 0: the general kernel on the schedule the preparation kernel left in the workspace;
+// 1, 2, 4 or 8: the single-launch kernel, one cluster of that many CTAs per (sequence, KV head, M tile).
+reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, int small_cluster, cudaStream_t st) {
     if (!h->attr_set) {
-        if (cudaFuncSetAttribute(attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(attn_sm100_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(attn_sm100_kernel<128, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<128, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<64, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytesSmall) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_sm100_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytesSmall) != cudaSuccess) {
             cudaGetLastError();
             return READER_ERR_CUDA;
         }
@@ -831,17 +1012,32 @@ reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t 
         m->q = p.q; m->qB = p.B; m->qT = p.T; m->qHq = p.Hq; m->qG = p.G; m->qD = p.D;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.sched.n_ctas);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = p.D == 128 ? Cfg<128>::kSmemBytes : Cfg<64>::kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // prologue overlaps the preparation kernel
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // prologue overlaps the kernel before it
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    auto kernel = p.D == 128 ? (p.valid_bits ? attn_sm100_kernel<128, true> : attn_sm100_kernel<128, false>)
-                             : (p.valid_bits ? attn_sm100_kernel<64, true> : attn_sm100_kernel<64, false>);
+    auto kernel = p.D == 128 ? (p.valid_bits ? attn_sm100_kernel<128, true, false> : attn_sm100_kernel<128, false, false>)
+                             : (p.valid_bits ? attn_sm100_kernel<64, true, false> : attn_sm100_kernel<64, false, false>);
+    if (small_cluster > 0) {
+        if (p.valid_bits) return READER_ERR_UNSUPPORTED;
+        const int n_mtiles = (p.T * p.G + kTileM - 1) / kTileM;
+        cfg.gridDim = dim3((unsigned)(p.B * p.Hkv * n_mtiles * small_cluster));
+        cfg.dynamicSmemBytes = p.D == 128 ? Cfg<128>::kSmemBytesSmall : Cfg<64>::kSmemBytesSmall;
+        kernel = p.D == 128 ? attn_sm100_kernel<128, false, true> : attn_sm100_kernel<64, false, true>;
+        if (small_cluster > 1) {
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = (unsigned)small_cluster;
+            attr[1].val.clusterDim.y = 1;
+            attr[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+        }
+    } else {
+        cfg.gridDim = dim3(p.sched.n_ctas);
+        cfg.dynamicSmemBytes = p.D == 128 ? Cfg<128>::kSmemBytes : Cfg<64>::kSmemBytes;
+    }
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p, pm->kmap, pm->vmap, m->ktmap, m->vtmap, m->qmap);
     if (e != cudaSuccess) {
         cudaGetLastError();

@@ -17,6 +17,6 @@ struct Sm100Host {
 reader_status sm100_host_init(Sm100Host *h, int device);
 void sm100_host_destroy(Sm100Host *h);
 bool sm100_supports(const Sm100Host *h, const AttnParams &p, float softmax_scale);
-reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, cudaStream_t st);
+reader_status launch_attn_sm100(Sm100Host *h, const AttnParams &p, int small_cluster, cudaStream_t st);
 
 }  // namespace reader

@@ -28,6 +28,7 @@ def rd():
 
 
 def gpu_attn(rd, w, kernel=0, pre_encode=False, want_lse=True):
+    """kernel: 0 automatic, 1 CUDA-core, 2 tensor-core on the three-launch path, 3 tensor-core as a single launch."""
     from paper_2508_09072_b200 import binding
     d = binding.to_device(w, with_logits=False)
     rd.set_attn_kernel(kernel)
@@ -39,10 +40,12 @@ def gpu_attn(rd, w, kernel=0, pre_encode=False, want_lse=True):
     # scratch that a kernel reads without having written it must show: fill it with NaN patterns
     ws = rd.workspace(max(w.batch, 1), w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
     ws.fill_(0xFF)
-    out, status = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out, lse=lse,
-                                 workspace=ws)
-    torch.cuda.synchronize()
-    rd.set_attn_kernel(0)
+    try:
+        out, status = rd.verify_attn(d.q, d.k_tree, d.v_tree, d.cache, d.parent, w.scale, anc_mask=anc, out=out, lse=lse,
+                                     workspace=ws)
+        torch.cuda.synchronize()
+    finally:
+        rd.set_attn_kernel(0)
     o = W.bf16_bits_to_f32(binding.bf16_bits(out)).astype(np.float64)
     return o, status.cpu().numpy(), (lse.cpu().numpy().astype(np.float64) if want_lse else None)
 
@@ -107,7 +110,7 @@ def test_tree_encode_matches_oracle(rd, T):
 
 
 # ------------------------------------------------------------------------------------ attention
-@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("kernel", [0, 1, 2, 3])
 @pytest.mark.parametrize("name", W.WORKLOADS)
 def test_attn_named_workloads_small(rd, name, kernel):
     w = W.make(name, with_logits=False, reduced=(name != "c1"))
@@ -128,10 +131,12 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("kernel", [0, 1, 2, 3])
 @pytest.mark.parametrize("case", range(len(SHAPES)))
 def test_attn_shapes_and_ragged_lengths(rd, case, kernel):
     T, Hq, Hkv, D, lens = SHAPES[case]
+    if kernel >= 2 and 128 % (Hq // Hkv) != 0:
+        pytest.skip("group of 3: CUDA-core kernel only")
     w = W.build_workload("s", 900 + case, list(lens), T, Hq, Hkv, D,
                          lambda r: W.capped_recursive_tree(r, T, 12, 4), max_path=12, vocab=16,
                          shuffle_pages=True, with_logits=False, spare_pages=3)
@@ -139,9 +144,11 @@ def test_attn_shapes_and_ragged_lengths(rd, case, kernel):
     check_attn(w, got, status, lse)
 
 
-def test_attn_random_shapes(rd):
+@pytest.mark.parametrize("kernel", [0, 2, 3])
+def test_attn_random_shapes(rd, kernel):
     """Seeded random shapes: tree size, GQA group (1..16, so 1 to 16 M tiles per KV stream), head
-    dimension, batch and ragged committed lengths (empty caches and exact page multiples included)."""
+    dimension, batch and ragged committed lengths (empty caches and exact page multiples included), through
+    the automatic choice, the three-launch path alone and the single-launch path alone."""
     rng = np.random.default_rng(20250809)
     for case in range(28):
         T = int(rng.choice([1, 2, 3, 7, 16, 31, 32, 33, 63, 64, 65, 100, 127, 128]))
@@ -153,7 +160,7 @@ def test_attn_random_shapes(rd):
         w = W.build_workload("r", 5000 + case, lens, T, G * Hkv, Hkv, D,
                              lambda r: W.capped_recursive_tree(r, T, 12, 4) if T > 1 else np.array([-1], np.int32),
                              max_path=12, vocab=16, shuffle_pages=True, with_logits=False, spare_pages=2)
-        got, status, lse = gpu_attn(rd, w, kernel=0, pre_encode=bool(case & 1))
+        got, status, lse = gpu_attn(rd, w, kernel=kernel, pre_encode=bool(case & 1))
         try:
             check_attn(w, got, status, lse)
         except AssertionError as e:
@@ -217,6 +224,42 @@ def test_attn_scheduler_extremes(rd, case):
     check_attn(w, got, status, lse)
 
 
+SINGLE_LAUNCH = [
+    # B, T, G, Hkv, D, lens: cluster sizes 8, 4, 2, 1 (by the number of units) and shares of many tiles
+    (1, 64, 4, 8, 128, (4096,)),            # C2's shape: 16 units, clusters of 8
+    (1, 16, 1, 8, 64, (512,)),              # C1's shape
+    (2, 32, 4, 8, 128, (3000, 1)),          # 16 units, one nearly empty sequence: shares without any tile
+    (4, 33, 4, 8, 128, (1500, 700, 64, 0)), # 64 units: clusters of 4
+    (9, 32, 4, 8, 128, (900, 100, 333, 64, 65, 0, 2000, 129, 640)),    # 72 units: clusters of 4
+    (3, 128, 16, 3, 128, (700, 300, 50)),   # 16 M tiles per KV stream: 144 units, clusters of 2
+    (30, 8, 2, 8, 64, (150,) * 30),         # 240 units: one CTA each, no merge
+]
+
+
+@pytest.mark.parametrize("case", range(len(SINGLE_LAUNCH)))
+def test_attn_single_launch_path(rd, case):
+    """reader_set_attn_kernel(3): checks, attention and merge in one launch, clusters of 1 to 8 CTAs per unit."""
+    B, T, G, Hkv, D, lens = SINGLE_LAUNCH[case]
+    w = W.build_workload("sl", 8800 + case, list(lens), T, G * Hkv, Hkv, D, lambda r: W.capped_recursive_tree(r, T, 12, 4),
+                         max_path=12, vocab=16, shuffle_pages=True, with_logits=False, spare_pages=1)
+    for pre in (False, True):
+        got, status, lse = gpu_attn(rd, w, kernel=3, pre_encode=pre)
+        check_attn(w, got, status, lse)
+    ref, _, _ = gpu_attn(rd, w, kernel=2)
+    assert np.abs(got - ref).max() <= 2 ** -6
+
+
+def test_attn_single_launch_path_refuses_what_does_not_fit_one_wave(rd):
+    from paper_2508_09072_b200 import binding
+    w = W.build_workload("sl", 8899, [10] * 300, 4, 2, 2, 64, lambda r: W.capped_recursive_tree(r, 4, 3, 2), max_path=3,
+                         vocab=16, shuffle_pages=True, with_logits=False)
+    with pytest.raises(binding.ReaderError) as e:
+        gpu_attn(rd, w, kernel=3)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    got, status, lse = gpu_attn(rd, w, kernel=0)
+    check_attn(w, got, status, lse)
+
+
 def test_attn_empty_batch_is_a_no_op(rd):
     from paper_2508_09072_b200 import binding
     w = W.make("c1", with_logits=False)
@@ -247,14 +290,15 @@ def test_attn_status_words_and_poisoned_tail(rd):
     pg = w.page_table[0, 1]
     w.k_pool[pg, :, 36:, :] = 0x7FC0                     # NaN / inf beyond seq_len 100 on its last page
     w.v_pool[pg, :, 36:, :] = 0x7F80
-    for kernel in (0, 1):
+    for kernel in (0, 1, 2, 3):
         got, status, lse = gpu_attn(rd, w, kernel=kernel)
         assert status.tolist() == [0, oracle.BAD_TREE, oracle.BAD_PAGE, 0]
         assert not got[1].any() and not got[2].any() and not lse[1].any() and not lse[2].any()
         check_attn(w, got, status, lse)
     w.seq_lens[3] = w.max_pages * 64 + 1
-    got, status, _ = gpu_attn(rd, w)
-    assert status[3] == oracle.CAPACITY and not got[3].any()
+    for kernel in (2, 3):
+        got, status, _ = gpu_attn(rd, w, kernel=kernel)
+        assert status[3] == oracle.CAPACITY and not got[3].any()
 
 
 def test_attn_shared_prefix_equals_duplicated_prefix(rd):
@@ -707,7 +751,7 @@ def test_multi_layer_step_in_one_graph_matches_oracle_layer_by_layer(rd):
         np.testing.assert_array_equal(slots.cpu().numpy(), com["slots"])
 
 
-@pytest.mark.parametrize("kernel", [1, 2])
+@pytest.mark.parametrize("kernel", [1, 2, 3])
 def test_prepare_once_then_every_layer(rd, kernel):
     """reader_verify_prepare + reader_verify_attn_prepared per layer against the oracle, one rejected
     sequence included: its rows must be zero in every layer's output."""
@@ -755,7 +799,7 @@ def test_error_flag_in_the_workspace_reaches_every_status_word_and_zeroes_the_ou
     w = W.make("c3", reduced=True, with_logits=False)
     d = binding.to_device(w, with_logits=False)
     ws = rd.workspace(w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, w.head_dim)
-    for kernel in (2, 1):
+    for kernel in (2, 1, 3):
         rd.set_attn_kernel(kernel)
         try:
             status, _ = rd.verify_prepare(d.cache, d.parent, w.n_q_heads, workspace=ws)
