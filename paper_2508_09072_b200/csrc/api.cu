@@ -554,7 +554,7 @@ reader_status reader_kv_rearrange(reader_ctx *ctx, void *k, void *v, int32_t bat
     if (batch == 0) return READER_OK;
     if (!k || !v || !valid || !lengths_out || batch < 0 || n_kv_heads < 1 || capacity < 1 || !aligned16(k) || !aligned16(v))
         return READER_ERR_INVALID_ARG;
-    if (head_dim < 8 || head_dim % 8 != 0 || head_dim > 256) return READER_ERR_UNSUPPORTED;   // 64 rows are staged in 48 KB
+    if (head_dim < 8 || head_dim % 8 != 0 || head_dim > 256) return READER_ERR_UNSUPPORTED;   // a chunk of at least 64 rows is staged in 40 KB
     if (reader_status st = check_device(ctx)) return st;
     launch_kv_rearrange(static_cast<__nv_bfloat16 *>(k), static_cast<__nv_bfloat16 *>(v), batch, n_kv_heads, capacity,
                         head_dim, valid, lengths_out, (cudaStream_t)stream);
