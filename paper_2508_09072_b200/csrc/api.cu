@@ -216,7 +216,7 @@ reader_status run_verify_attn(reader_ctx *ctx, AttnParams p, const reader_kv_cac
     // launches of mostly latency on the general path.  It takes one launch instead: every unit
     // (sequence, KV head, M tile) gets a cluster of up to 8 CTAs that checks the sequence, shares the unit's
     // tiles and merges the shares in distributed shared memory.  Chosen when the clusters fit the GPU in one
-    // wave and a share is at most kSmallTilesPerCta tiles (judged by the page table's width: lengths live on
+    // wave and a share is at most kSmallTilesPerCta tiles (going by the page table's width: lengths live on
     // the device); reader_set_attn_kernel(3) takes it whenever the clusters fit.
     int small_cluster = 0;
     p.parent = tree->parent;

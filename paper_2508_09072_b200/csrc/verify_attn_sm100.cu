@@ -320,7 +320,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         mine.h = (unit / n_mtiles) % p.Hkv;
         mine.b = unit / (n_mtiles * p.Hkv);
         // Only the committed length is needed to start loading: the checks of the tree and of the page ids run
-        // in the softmax warps (below) while the first tiles are on their way, and their verdict is used at the
+        // in the softmax warps (below) while the first tiles are on their way, and their outcome is used at the
         // end.  (A page id outside the pool makes a tile load read the fill value, never a fault.)
         const int L = p.seq_lens[mine.b];
         const bool len_ok = L >= 0 && (int64_t)L <= (int64_t)p.max_pages * kPage;
