@@ -776,7 +776,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
     tc_fence_before();
     __syncthreads();
     if constexpr (kSmall) {
-        // The shares of a unit meet here: CTA r of the cluster merges rows 128 r / size .. of the unit out of
+        // The shares of a unit meet here: CTA r of the cluster merges its r-th part of the unit's rows out of
         // every CTA's partial (m* = max m_s, l* = sum l_s 2^(m_s - m*), O = sum O_s 2^(m_s - m*) / l*)
         // and writes them.  A rejected sequence, or a CTA that gave up on a bounded wait, gets zero rows.
         const bool multi = cl_size > 1;
@@ -790,7 +790,9 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             cluster_wait_acquire();
         }
         if (warp < kSoftmaxWarps && (multi || reject != 0 || gave_up)) {
-            const int rows_per = kTileM / (int)cl_size;
+            // the unit's real rows (a small tree fills only the first of the 128) are dealt out evenly
+            const int rows_real = min(kTileM, p.T * p.G - mine.mt * kTileM);
+            const int rows_per = (rows_real + (int)cl_size - 1) / (int)cl_size;
             const bool has_cols = lane * 4 < D;
             const int cta0 = cta - (int)cl_rank;   // the cluster's first CTA: share q lies in partial slot cta0 + q
             int peer_flag = 0;   // consumed after the first row's loads have been issued: one round trip to L2, not two
@@ -799,7 +801,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             for (int rr = warp; rr < rows_per; rr += kSoftmaxWarps) {
                 const int row = (int)cl_rank * rows_per + rr;
                 const int grow = mine.mt * kTileM + row;
-                if (grow >= p.T * p.G) continue;
+                if (row >= rows_real) continue;
                 float mstar = -INFINITY, lstar = 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 bool bad = reject != 0 || gave_up;
