@@ -18,15 +18,16 @@
 //               tile a single issuer was the bottleneck of the whole kernel.
 //   warps 0-7   softmax: warp w owns the 16 query rows 32 (w % 4) + 16 (w / 4) .. + 15 (TMEM lanes), a
 //               quad of threads per row pair (rows r and r + 8), so a thread handles 16 of a row's 64
-//               scores and a row's maximum costs two shuffles.  (With one thread per row, 4 warps, a
-//               tile's softmax took ~1350 cycles and sat between the value product of tile i-1 and the
-//               score product of tile i+1 on the critical path; eight warps halve that latency and
-//               give each scheduler four warps to hide it.)  Scores come from TMEM, the ancestor
+//               scores and a row's maximum costs two shuffles.  Scores come from TMEM, the ancestor
 //               bitmask / length mask is applied, the running maximum is raised only when it grows
 //               by more than 2^8 (the accumulator in TMEM is rescaled then), probabilities (bf16
-//               pairs) are written over the scores they came from and are the value product's A
-//               operand straight from tensor memory.  The same threads write O (or an (m, l, O)
-//               partial) at the end of a segment.
+//               pairs) go to one of two probability tiles in TMEM and are the value product's A
+//               operand straight from there.  The same threads write O (or an (m, l, O) partial) at
+//               the end of a segment.
+//
+// The same kernel has a second form (kSmall) for calls with few units, launched alone: one thread-block
+// cluster per unit whose CTAs check the sequence, share the unit's tiles and merge their shares after the
+// cluster's hardware barrier (see where kSmall is tested below).
 //
 // Bytes beyond a sequence's length or the tree's end can never reach a product: scores there are
 // replaced by -inf, and the value product skips 16-key slices past the end and zeroes the tail of
@@ -45,8 +46,8 @@
 // alternate strictly (the score product of tile i+1 needs every softmax thread's arrival for tile i, which
 // comes after that thread saw tile i), so one barrier each is enough; p_full and pv_done, which warps
 // reach at different times, exist once per probability tile: the waiter for tile i on barrier i & 1 knows
-// that tile i-2 is complete and that tile i+2 cannot have been issued.  Every wait is bounded: after one second without progress a CTA raises the error flag in the workspace,
-// stops waiting and runs to its end.
+// that tile i-2 is complete and that tile i+2 cannot have been issued.  Every wait is bounded: after one
+// second without progress a CTA raises the error flag in the workspace, stops waiting and runs to its end.
 #include <cuda.h>
 
 #include <new>
