@@ -53,6 +53,34 @@ def test_noalloc_accept_equals_accept_on_two_calls_in_a_row():
         rd.close()
 
 
+def test_noalloc_accept_from_a_second_context_on_another_stream():
+    """The scratch array belongs to the library, not to a context: a second context, calling on a stream of its
+    own after the first context's calls have finished, finds the array with someone else's pairs in it and must
+    still return the oracle's result."""
+    from paper_2508_09072_b200 import binding
+    w = W.build_workload("na3", 4244, [20] * 7, 23, 2, 1, 64, lambda r: W.capped_recursive_tree(r, 23, 6, 3),
+                         max_path=6, vocab=30011, shuffle_pages=False)
+    first, second = binding.Reader(0), binding.Reader(0)
+    try:
+        _both(first, w)                                            # leaves its pairs behind (synchronised inside)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            parent = torch.from_numpy(w.parent).cuda()
+            tok = torch.from_numpy(w.node_tokens).cuda()
+            logits = torch.from_numpy(w.logits).cuda()
+            got = second.accept_noalloc(parent, tok, w.max_path, logits)
+            side.synchronize()
+        got = {k: v.cpu().numpy() for k, v in got.items()}
+        tgt = oracle.argmax(w.logits)
+        np.testing.assert_array_equal(got["target_ids"], tgt)
+        want = oracle.accept(w.parent, w.node_tokens, tgt, w.max_path)
+        for k in ("path", "n_acc", "bonus", "status"):
+            np.testing.assert_array_equal(got[k], want[k], err_msg=k)
+    finally:
+        first.close()
+        second.close()
+
+
 def test_noalloc_accept_refuses_what_its_array_cannot_hold():
     from paper_2508_09072_b200 import binding
     rd = binding.Reader(0)
