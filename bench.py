@@ -623,7 +623,9 @@ def run_ours(args):
                               "is timed, the median block is reported"},
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "blocks": ne,
                     "ms_per_step": ms_e2e_block / K},
-            "gpu_launches": LAUNCHES_PER_ATTN_CALL * K * n_blocks, "clocks": clocks, "roofline": roof,
+            # C1 and C2 take the single-launch form of the attention kernel (unless a kernel was forced)
+            "gpu_launches": (1 if (args.workload in ("c1", "c2") and args.kernel in (0, 3)) else LAUNCHES_PER_ATTN_CALL) * K * n_blocks,
+            "clocks": clocks, "roofline": roof,
             "whole_step": {"ms_per_step": t_step, "tokens_per_s": tokens / (t_step * 1e-3), "launches_per_step": LAUNCHES_PER_STEP,
                            "steps": Ks, "note": "reader_verify_attn (masks encoded inside) + reader_accept_commit from logits, "
                                                 "back to back; reported beside the metric, not folded into it"},
