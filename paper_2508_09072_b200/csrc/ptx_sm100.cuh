@@ -209,6 +209,15 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// True in exactly one lane of a converged warp.  Code that issues tcgen05.mma from one thread should branch
+// on this rather than on a lane number: with `if (lane == 0)` around the eight score MMAs of a tile one
+// instruction started every 110-160 cycles; behind elect.sync one starts every 48 (N = 64) or 64 (N = 128)
+// cycles, which is the tensor pipe's own pace (measured on this GPU).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.b32 %0, 1, 0, q;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 // The mbarrier gets one arrival when every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

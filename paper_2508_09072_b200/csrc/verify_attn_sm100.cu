@@ -439,7 +439,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 // the score tile is free as soon as every softmax thread holds the previous scores in registers
                 wait(bar(&bars->s_empty), (i & 1) ^ 1, abort_s, p.error_flag);
                 tc_fence_after();
-                if (lane == 0) {
+                __syncwarp();
+                if (elect_one()) {
                     const uint64_t kd = descK + (uint64_t)((stage * C::kTileBytes) >> 4);
 #pragma unroll
                     for (int hf = 0; hf < C::kHalves; ++hf)
@@ -527,7 +528,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                         __syncwarp();
                     }
                 }
-                if (lane == 0) {
+                __syncwarp();
+                if (elect_one()) {
                     const uint64_t vd = descV + (uint64_t)((stage * C::kTileBytes) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
