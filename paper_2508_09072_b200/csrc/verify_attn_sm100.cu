@@ -227,7 +227,8 @@ __device__ __forceinline__ void load_tile(const AttnParams &p, const TileCursor<
                                           uint64_t stream_policy, int first_streamed_tile) {
     using C = Cfg<D>;
     const int page = c.page();
-    if (lane != 0) return;
+    __syncwarp();
+    if (!elect_one()) return;   // (as for the MMA issuers: behind elect.sync the copies are issued back to back)
     mbar_arrive_expect_tx(full, C::kTileBytes);
     if (c.t < c.sg.npages) {
         int row;
@@ -375,7 +376,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, q_w, w_end, lane);
                 q_w += sg.span;
                 if (sg.tile_end <= sg.tile_begin) continue;   // no real tile: no query tile
-                if (lane == 0) {
+                __syncwarp();
+                if (elect_one()) {
                     const uint32_t full = bar(&bars->q_full);
                     mbar_arrive_expect_tx(full, C::kQBytes);
 #pragma unroll
