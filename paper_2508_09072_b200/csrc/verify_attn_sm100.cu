@@ -13,9 +13,9 @@
 //               segment's last score product is done.  A K slot is free again as soon as its score
 //               product has run, long before the tile's value product, so key loads run far ahead.
 //   warp 9      issues S[i] = Q K[i]^T as soon as K[i] has landed and the score tile is free
-//   warp 10     issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Two issuing warps because
-//               one thread can start a tcgen05.mma only every ~120 cycles: with 8 + 4 of them per
-//               tile a single issuer was the bottleneck of the whole kernel.
+//   warp 10     issues O += P[j] V[j] as soon as P[j] and V[j] are ready.  Both issuers (and the producer)
+//               issue from the lane elect.sync picks: under `if (lane == 0)` one tcgen05.mma started
+//               only every 110-160 cycles, behind elect.sync one starts every 48-64.
 //   warps 0-7   softmax: warp w owns the 16 query rows 32 (w % 4) + 16 (w / 4) .. + 15 (TMEM lanes), a
 //               quad of threads per row pair (rows r and r + 8), so a thread handles 16 of a row's 64
 //               scores and a row's maximum costs two shuffles.  Scores come from TMEM, the ancestor
@@ -421,8 +421,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ score-product issuer
-        // (one thread can start a tcgen05.mma only every ~120 cycles, so the two kinds of product
-        // are issued by two warps)
+        // (its own warp, so that a tile's value product never queues behind the next tile's score product)
         constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kPage, false, false);
         // descriptors differ only in their start-address field (bytes >> 4), so each operand's
         // descriptor is one addition away from a base built once
