@@ -63,9 +63,14 @@ __device__ __forceinline__ int effective_ctas(int n_launched, int W) {
     return max(1, min(n_launched, (W + kMinTilesPerCta - 1) / kMinTilesPerCta));
 }
 
+// floor(c * W / n) for 0 <= c <= n <= 2^15 and 0 <= W < 2^31, in 32-bit arithmetic: c W = c n (W / n) + c (W % n).
+// (A 64-bit division is a few hundred dependent instructions on this GPU; the thread that located a cut
+// unit's last partial with three of them held its CTA up for 2.4 us at every such segment.)
+__device__ __forceinline__ int mul_div(int c, int W, int n) { return c * (W / n) + (c * (W % n)) / n; }
+
 // First tile of CTA c's range; c >= n_ctas (a CTA left without work) gets W.
 __device__ __forceinline__ int range_begin(int c, int n_ctas, int W) {
-    return c >= n_ctas ? W : (int)(((int64_t)c * W) / n_ctas);
+    return c >= n_ctas ? W : mul_div(c, W, n_ctas);
 }
 
 // Largest b with seq_tile_start[b] <= w (w < W).
@@ -162,8 +167,8 @@ __device__ __forceinline__ Segment segment_at_warp(const Sched &s, const WarpSch
 
 // Lane (of n_ctas lanes) whose range contains flat tile w.
 __device__ __forceinline__ int cta_of_tile(int w, int n_ctas, int W) {
-    int c = (int)(((int64_t)w * n_ctas) / W);
-    if (c >= n_ctas) c = n_ctas - 1;
+    int c = (int)((float)w * (float)n_ctas / (float)W);   // a first guess; the loops below make it exact
+    c = max(0, min(c, n_ctas - 1));
     while (c + 1 < n_ctas && range_begin(c + 1, n_ctas, W) <= w) ++c;
     while (c > 0 && range_begin(c, n_ctas, W) > w) --c;
     return c;
@@ -207,7 +212,7 @@ __device__ __forceinline__ LaneRange lane_range(const Sched &s, int B, int lane,
         const int st = lane / k, j = lane - st * k;
         if (st >= n_streams) return LaneRange{W, W};
         stream_span(s, st, start, len);
-        return LaneRange{start + (int)(((int64_t)j * len) / k), start + (int)(((int64_t)(j + 1) * len) / k)};
+        return LaneRange{start + mul_div(j, len, k), start + mul_div(j + 1, len, k)};
     }
     const int q = (n_streams + n_lanes - 1) / n_lanes;
     const int s0 = lane * q, s1 = min(n_streams, s0 + q);
@@ -226,10 +231,10 @@ __device__ __forceinline__ int lane_of_entry(const Sched &s, int B, const Segmen
     if (n_lanes >= n_streams) {
         const int k = n_lanes / n_streams;
         const int len = g.ntiles + kUnitOverhead, pos = w - g.unit_w0;
-        int j = (int)(((int64_t)pos * k) / len);
-        if (j >= k) j = k - 1;
-        while (j + 1 < k && (int)(((int64_t)(j + 1) * len) / k) <= pos) ++j;
-        while (j > 0 && (int)(((int64_t)j * len) / k) > pos) --j;
+        int j = (int)((float)pos * (float)k / (float)len);   // a first guess, made exact below
+        j = max(0, min(j, k - 1));
+        while (j + 1 < k && mul_div(j + 1, len, k) <= pos) ++j;
+        while (j > 0 && mul_div(j, len, k) > pos) --j;
         return st * k + j;
     }
     return st / ((n_streams + n_lanes - 1) / n_lanes);

@@ -332,8 +332,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         mine.ntiles = n;
         mine.npages = npages;
         mine.len = L;
-        mine.tile_begin = (int)(((int64_t)cl_rank * n) / cl_size);
-        mine.tile_end = (int)(((int64_t)(cl_rank + 1) * n) / cl_size);
+        mine.tile_begin = mul_div((int)cl_rank, n, (int)cl_size);
+        mine.tile_end = mul_div((int)cl_rank + 1, n, (int)cl_size);
         mine.full = cl_size == 1;
         mine.slot = cta;
         w_end = mine.tile_end - mine.tile_begin;
@@ -463,9 +463,20 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         const uint64_t descV = smem_desc_sw128(sV, C::kHalfRowsKV, 1024);
         int i = 0;
         int w = w_begin;
+        // This warp also leaves the note the combine kernel needs about a unit this CTA starts without finishing
+        // it (at most one per CTA): it has time to spare at the start of a segment, the softmax warps do not.
+        // (A CTA that gives up on a wait may skip a note: the combine kernel then reports the timeout instead.)
+        if constexpr (!kSmall) {
+            if (lane == 0) p.split_desc[cta].b = -1;
+            __syncwarp();
+        }
         while (w < w_end && !*abort_s) {
             const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, w, w_end, lane);
             const int n = sg.tile_end - sg.tile_begin;
+            if constexpr (!kSmall) {
+                if (lane == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
+                __syncwarp();
+            }
             w += sg.span;
             if (n <= 0) continue;
             const int L = sg.len;
@@ -552,6 +563,7 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
         constexpr uint32_t kNegInf = 0xff800000u;
         int it = 0;
         int w = w_begin;
+        const int lg_G = 31 - __clz(p.G);
         bool tree_ok = true;
         if constexpr (kSmall) {
             // the checks the preparation kernel makes for large calls: parent[0] = -1 and 0 <= parent[j] < j; every
@@ -571,25 +583,21 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxWarps * 32) : "memory");
             tree_ok = (*reinterpret_cast<volatile int32_t *>(&bars->reject) & 1) == 0;
         }
-        if constexpr (!kSmall) {
-            if (tid == 0) p.split_desc[cta].b = -1;
-        } else if (w_end == 0 && cpair == 0) {
+        if (kSmall && w_end == 0 && cpair == 0) {
             // no tile fell to this CTA: its share of the unit is the empty partial
             *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)cta * kTileM + row_a) * 2) = make_float2(-INFINITY, 0.f);
             *reinterpret_cast<float2 *>(p.partial_ml + ((size_t)cta * kTileM + row_b) * 2) = make_float2(-INFINITY, 0.f);
         }
         while (w < w_end) {
             const Segment sg = seg_at<kSmall, kPadded>(p, wsched, mine, cta, w, w_end, lane);
-            if constexpr (!kSmall) {
-                if (tid == 0) record_split(p.split_desc, p.sched, p.B, cw.n_lanes, sg, cta, W);
-            }
             w += sg.span;
             if (sg.tile_end <= sg.tile_begin) continue;
             const int L = sg.len;
             const int grow_a = sg.mt * kTileM + row_a, grow_b = grow_a + 8;
             const bool ok_a = grow_a < p.T * p.G, ok_b = grow_b < p.T * p.G;
-            const int j_a = ok_a ? grow_a / p.G : 0, j_b = ok_b ? grow_b / p.G : 0;
-            const int hq_a = sg.h * p.G + (ok_a ? grow_a % p.G : 0), hq_b = sg.h * p.G + (ok_b ? grow_b % p.G : 0);
+            // (G divides 128, so it is a power of two: shifts, not divisions, on the path into a segment)
+            const int j_a = ok_a ? grow_a >> lg_G : 0, j_b = ok_b ? grow_b >> lg_G : 0;
+            const int hq_a = sg.h * p.G + (ok_a ? grow_a & (p.G - 1) : 0), hq_b = sg.h * p.G + (ok_b ? grow_b & (p.G - 1) : 0);
 
             uint64_t anc_a[2] = {0, 0}, anc_b[2] = {0, 0};
             if (kSmall && p.anc == nullptr) {   // no encoded masks at hand: walk the parent array (in shared memory)
