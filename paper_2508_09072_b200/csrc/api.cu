@@ -30,7 +30,7 @@ WsLayout ws_layout(const reader_ctx *ctx, int B, int T, int D) {
     size_t at = 0;
     auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes); return o; };
     const size_t slots = 2 * (size_t)max_ctas(ctx);
-    w.error_flag = take(sizeof(int32_t));
+    w.error_flag = take(2 * sizeof(int32_t));   // the flag; behind it the preparation kernel's "blocks done" counter
     w.seq_tile_start = take(sizeof(int32_t) * ((size_t)B + 1));
     w.seq_ntiles = take(sizeof(int32_t) * (size_t)B);
     w.seq_npages = take(sizeof(int32_t) * (size_t)B);

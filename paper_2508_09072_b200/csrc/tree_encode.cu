@@ -52,10 +52,14 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
                                                        __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
                                                        int Hq, int D) {
     __shared__ int32_t par[32][kMaxNodes];
+    __shared__ int s_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // A large batch is shared by several blocks, 32 sequences (one per warp) at a time each; the block that
+    // finishes last (a counter in the workspace, zeroed by the host before the launch) makes the prefix sums.
+    const int gwarp = blockIdx.x * 32 + warp, n_gwarps = gridDim.x * 32;
     pdl_launch_dependents();   // the attention kernel may set itself up meanwhile
     pdl_wait();                // this kernel itself is launched ahead of its predecessor's end
-    if (threadIdx.x == 0) *error_flag = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *error_flag = 0;
     const bool padded = pd.valid != nullptr;
     const int extent = padded ? *pd.extent : 0;
     const bool extent_ok = extent >= 0 && extent <= pd.cap;
@@ -63,7 +67,7 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
         // 16 mask bytes -> 16 bits; pieces from the extent on (up to the end of its tile) read as zero
         const int pieces = ((extent + kPage - 1) / kPage) * (kPage / 16);
         const bool vec = (pd.cap % 16 == 0) && (reinterpret_cast<uintptr_t>(pd.valid) % 16 == 0);
-        for (int i = threadIdx.x; i < B * pieces; i += blockDim.x) {
+        for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < B * pieces; i += gridDim.x * blockDim.x) {
             const int b = i / pieces, c = i - b * pieces;
             const int first = c * 16, n = min(16, extent - first);   // n <= 0: past the extent
             uint32_t bits = 0;
@@ -85,7 +89,7 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
             reinterpret_cast<uint16_t *>(pd.bits + (size_t)b * pd.bits_per_seq)[c] = (uint16_t)bits;
         }
     }
-    for (int b = warp; b < B; b += 32) {
+    for (int b = gwarp; b < B; b += n_gwarps) {
         for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];
         __syncwarp();
         int st = warp_tree_valid(par[warp], T, lane) ? READER_OK : READER_ERR_BAD_TREE;
@@ -132,12 +136,22 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
         __syncwarp();
     }
     __syncthreads();
+    if (gridDim.x > 1) {
+        if (threadIdx.x == 0) {
+            __threadfence();   // this block's seq_ntiles before its count
+            s_last = atomicAdd(error_flag + 1, 1) == (int)gridDim.x - 1;
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    }
     if (warp == 0) {
         int carry = 0;
         if (lane == 0) seq_tile_start[0] = 0;
         for (int base = 0; base < B; base += 32) {
             int b = base + lane;
-            int v = b < B && seq_ntiles[b] > 0 ? (seq_ntiles[b] + kUnitOverhead) * units_per_seq : 0;
+            const int nt = b < B ? __ldcg(seq_ntiles + b) : 0;   // (possibly another block's: not through L1)
+            int v = nt > 0 ? (nt + kUnitOverhead) * units_per_seq : 0;
             int incl = v;
             for (int d = 1; d < 32; d <<= 1) {
                 int t = __shfl_up_sync(0xffffffffu, incl, d);
@@ -153,7 +167,13 @@ void launch_prepare(const reader_kv_cache &c, const PaddedIn &padded, const int3
                     int units_per_seq, uint64_t *anc_out, int32_t *seq_tile_start, int32_t *seq_ntiles,
                     int32_t *seq_npages, int32_t *status, int32_t *error_flag, __nv_bfloat16 *out, float *lse,
                     int Hq, int D, cudaStream_t st) {
-    launch_pdl(prepare_kernel, dim3(1), dim3(1024), 0, st, padded, c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages,
+    // one block up to 64 sequences (two rounds of its 32 warps); beyond that a block per 32 sequences, up to 64 blocks
+    int blocks = 1;
+    if (B > 64) {
+        blocks = (B + 31) / 32 < 64 ? (B + 31) / 32 : 64;
+        cudaMemsetAsync(error_flag + 1, 0, sizeof(int32_t), st);   // the "blocks done" counter behind the flag
+    }
+    launch_pdl(prepare_kernel, dim3(blocks), dim3(1024), 0, st, padded, c.page_table, c.seq_lens, c.max_pages_per_seq, c.num_pages,
                parent, B, T, n_tree_tiles, units_per_seq, anc_out, seq_tile_start, seq_ntiles, seq_npages, status,
                error_flag, out, lse, Hq, D);
 }

@@ -282,6 +282,25 @@ def test_attn_many_short_sequences_and_widened_trees(rd):
     check_attn(w, got, status, lse)
 
 
+def test_attn_batch_of_150_prepared_by_several_blocks(rd):
+    """Above 64 sequences the preparation (tree checks, masks, page checks, tile prefix sums) is shared by
+    several thread blocks; a bad tree and a bad page id in the middle must still zero exactly their sequences."""
+    rng = np.random.default_rng(79)
+    lens = rng.integers(0, 130, size=150)
+    w = W.build_workload("s", 80, lens, 9, 4, 2, 64, lambda r: W.capped_recursive_tree(r, 9, 4, 3), max_path=4,
+                         vocab=16, shuffle_pages=True, with_logits=False)
+    w.parent[70, 4] = 6                                   # forward parent
+    victim = int(np.argmax(lens))
+    w.page_table[victim, 0] = w.num_pages + 1             # page id outside the pool
+    for kernel in (0, 1):
+        got, status, lse = gpu_attn(rd, w, kernel=kernel)
+        want = [0] * 150
+        want[70] = oracle.BAD_TREE
+        want[victim] = oracle.BAD_PAGE
+        assert status.tolist() == want
+        check_attn(w, got, status, lse)
+
+
 def test_attn_status_words_and_poisoned_tail(rd):
     w = W.build_workload("s", 81, [100, 70, 150, 64], 12, 8, 2, 128, lambda r: W.capped_recursive_tree(r, 12, 5, 3),
                          max_path=5, vocab=16, shuffle_pages=True, with_logits=False)
