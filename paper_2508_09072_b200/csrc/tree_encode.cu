@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
         }
     }
     for (int b = gwarp; b < B; b += n_gwarps) {
+        const int L = padded ? extent : seq_lens[b];   // (requested with the parents: one round trip, not two)
         for (int j = lane; j < T; j += 32) par[warp][j] = parent[(size_t)b * T + j];
         __syncwarp();
         int st = warp_tree_valid(par[warp], T, lane) ? READER_OK : READER_ERR_BAD_TREE;
@@ -102,7 +103,6 @@ __global__ void __launch_bounds__(1024) prepare_kernel(const PaddedIn pd,
                 anc_out[((size_t)b * T + j) * 2 + 1] = hi;
             }
         }
-        const int L = padded ? extent : seq_lens[b];
         int npages = 0;
         if (padded) {
             if (!extent_ok) st = READER_ERR_CAPACITY;   // whatever the tree: no sample can be served
