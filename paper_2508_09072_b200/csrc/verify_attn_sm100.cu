@@ -654,15 +654,18 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 xa0 = max3(xa0, f(20), f(21)); xa1 = max3(xa1, f(24), f(25));
                 xb0 = max3(xb0, f(22), f(23)); xb1 = max3(xb1, f(26), f(27));
                 float mx_a = max3(xa0, xa1, fmaxf(f(28), f(29))), mx_b = max3(xb0, xb1, fmaxf(f(30), f(31)));
-                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
-                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
-                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
-                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
-                const float mn_a = fmaxf(m_a, mx_a * p.scale_log2), mn_b = fmaxf(m_b, mx_b * p.scale_log2);
+                // A row's maximum rises (by more than 2^8) exactly if one of its four threads holds such a score, so
+                // the vote needs no exchange within the quad; the two shuffle rounds that give the row maxima
+                // themselves are paid only by the tiles that do raise one (a segment's first tile always does).
                 const bool first = t == sg.tile_begin;
-                const bool raise = __any_sync(0xffffffffu, mn_a > m_a + kRaiseMaxBy || mn_b > m_b + kRaiseMaxBy);
+                const bool raise = __any_sync(0xffffffffu, mx_a * p.scale_log2 > m_a + kRaiseMaxBy || mx_b * p.scale_log2 > m_b + kRaiseMaxBy);
                 float alpha_a = 1.f, alpha_b = 1.f;
                 if (raise || first) {
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+                    const float mn_a = fmaxf(m_a, mx_a * p.scale_log2), mn_b = fmaxf(m_b, mx_b * p.scale_log2);
                     alpha_a = (mn_a == -INFINITY) ? 1.f : ex2(m_a - mn_a);
                     alpha_b = (mn_b == -INFINITY) ? 1.f : ex2(m_b - mn_b);
                     m_a = mn_a; m_b = mn_b;
