@@ -599,21 +599,18 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             const int j_a = ok_a ? grow_a >> lg_G : 0, j_b = ok_b ? grow_b >> lg_G : 0;
             const int hq_a = sg.h * p.G + (ok_a ? grow_a & (p.G - 1) : 0), hq_b = sg.h * p.G + (ok_b ? grow_b & (p.G - 1) : 0);
 
-            uint64_t anc_a[2] = {0, 0}, anc_b[2] = {0, 0};
-            if (kSmall && p.anc == nullptr) {   // no encoded masks at hand: walk the parent array (in shared memory)
-                int lv;
-                if (ok_a && tree_ok) node_ancestors(par, p.T, j_a, anc_a[0], anc_a[1], lv);
-                if (ok_b && tree_ok) node_ancestors(par, p.T, j_b, anc_b[0], anc_b[1], lv);
-            } else {
-                if (ok_a) {
-                    anc_a[0] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 0];
-                    anc_a[1] = p.anc[((size_t)sg.b * p.T + j_a) * 2 + 1];
+            // The ancestor masks are fetched when a tree tile comes up (the last one or two tiles of a unit), not
+            // kept in eight registers through the committed tiles: the loop below runs at the register ceiling.
+            auto tree_mask = [&](int tree_tile, bool ok, int j) -> uint64_t {
+                if (!ok) return 0ull;
+                if (kSmall && p.anc == nullptr) {   // no encoded masks at hand: walk the parent array (in shared memory)
+                    uint64_t lo = 0, hi = 0;
+                    int lv;
+                    if (tree_ok) node_ancestors(par, p.T, j, lo, hi, lv);
+                    return tree_tile ? hi : lo;
                 }
-                if (ok_b) {
-                    anc_b[0] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 0];
-                    anc_b[1] = p.anc[((size_t)sg.b * p.T + j_b) * 2 + 1];
-                }
-            }
+                return p.anc[((size_t)sg.b * p.T + j) * 2 + tree_tile];
+            };
 
             float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // l: this thread's share of the row sums
             for (int t = sg.tile_begin; t < sg.tile_end; ++t, ++it) {
@@ -622,8 +619,8 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
                 if (t < sg.npages) {
                     vis_a = vis_b = visible_of<kPadded>(p, sg.b, t, L);
                 } else {
-                    vis_a = anc_a[t - sg.npages];
-                    vis_b = anc_b[t - sg.npages];
+                    vis_a = tree_mask(t - sg.npages, ok_a, j_a);
+                    vis_b = tree_mask(t - sg.npages, ok_b, j_b);
                 }
                 const int buf = it & 1;
                 wait(bar(&bars->s_full), it & 1, abort_s, p.error_flag);
