@@ -18,7 +18,8 @@
 //               only every 110-160 cycles, behind elect.sync one starts every 48-64.
 //   warps 0-7   softmax: warp w owns the 16 query rows 32 (w % 4) + 16 (w / 4) .. + 15 (TMEM lanes), a
 //               quad of threads per row pair (rows r and r + 8), so a thread handles 16 of a row's 64
-//               scores and a row's maximum costs two shuffles.  Scores come from TMEM, the ancestor
+//               scores and a row's maximum costs two shuffles (paid only when it rises: the vote on that
+//               uses the threads' own maxima).  Scores come from TMEM, the ancestor
 //               bitmask / length mask is applied, the running maximum is raised only when it grows
 //               by more than 2^8 (the accumulator in TMEM is rescaled then), probabilities (bf16
 //               pairs) go to one of two probability tiles in TMEM and are the value product's A
