@@ -359,10 +359,10 @@ attn_sm100_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, 
             prefetch_tensormap(&vtmap);
             prefetch_tensormap(&qmap);
         }
-        // pages are read exactly once when a KV head has a single M tile and nothing is shared (with a
-        // shared prefix the hint measured slightly slower, so it is left off there)
+        // pages are read exactly once when a KV head has a single M tile, except those of a shared prefix, which
+        // the other sequences' CTAs will ask for again: the hint goes on the private pages only
         const uint64_t stream_policy = l2_policy_evict_first();
-        const int first_streamed_tile = (p.sched.n_mtiles == 1 && p.shared_prefix_pages == 0) ? 0 : 0x7fffffff;
+        const int first_streamed_tile = p.sched.n_mtiles == 1 ? p.shared_prefix_pages : 0x7fffffff;
         TileCursor<kPadded, kSmall> kc, vc;
         kc.init(p, wsched, mine, cta, lane, w_begin, w_end);
         vc.init(p, wsched, mine, cta, lane, w_begin, w_end);
